@@ -1,0 +1,134 @@
+/*
+ * w4a8.h - C ABI of the B200 (sm_100a) W4A8 quantized linear layer.
+ *
+ * The operation is the paper's W4A8 scheme (Sec. 3.4, "Quantization": 4-bit weights,
+ * 8-bit activations, INT8 matrix multiply).  The paper fixes no bit layout, group
+ * size or rounding; this library uses:
+ *
+ *   weights      q_w[n,k] in 0..15; per (group of 128 consecutive k, output channel n)
+ *                one fp16 scale s_w[g,n] and one zero point z[g,n] in 0..15
+ *                (dequantised weight = s_w * (q_w - z))
+ *   activations  per token m: s_a[m] = fp16_rne(max_k |x[m,k]| / 127), saturating at 65504;
+ *                q_a[m,k] = clamp(round_half_even(x[m,k] / s_a[m]), -127, 127);
+ *                a token whose scale is 0 has all codes 0
+ *   partials     D[m,g,n] = sum_{k in g} q_w[n,k] q_a[m,k] - z[g,n] sum_{k in g} q_a[m,k]   (int32, exact)
+ *   output       y[m,n]   = bf16_rne( s_a[m] * sum_g s_w[g,n] * D[m,g,n] )   (fp32 accumulation over g)
+ *
+ * M tokens, K in-features, N out-features, G = K / group.  y = x W^T with W stored [N,K].
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller.  Inputs are only read,
+ *     outputs are fully overwritten.  Nothing is allocated or freed by the library.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Work is
+ *     enqueued on it; the host is never synchronised (w4a8_check_status excepted).
+ *   - Errors are reported by return value only.  After W4A8_ERR_CUDA the CUDA error is
+ *     left in place for cudaGetLastError().
+ *   - Shapes: group must be 128, K a multiple of 128, N a multiple of 128, M >= 0
+ *     (M == 0 returns W4A8_OK and enqueues nothing), otherwise W4A8_ERR_SHAPE.
+ *   - The device must be compute capability 10.x, otherwise W4A8_ERR_ARCH.
+ */
+#ifndef W4A8_H_
+#define W4A8_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    W4A8_OK = 0,
+    W4A8_ERR_NULL = 1,       /* a required pointer is NULL                                   */
+    W4A8_ERR_SHAPE = 2,      /* unsupported M, N, K or group                                 */
+    W4A8_ERR_ALIGN = 3,      /* a pointer misses its stated alignment                        */
+    W4A8_ERR_WORKSPACE = 4,  /* workspace_bytes < w4a8_workspace_bytes(M, N, K, group)       */
+    W4A8_ERR_ARCH = 5,       /* current device is not sm_100                                 */
+    W4A8_ERR_CUDA = 6,       /* a CUDA runtime/driver call failed                            */
+    W4A8_ERR_TIMEOUT = 7     /* a bounded device-side wait expired (seen via check_status)   */
+} w4a8_status;
+
+/* Which GEMM kernel family w4a8_gemm_path runs. */
+typedef enum {
+    W4A8_PATH_AUTO = 0,      /* dispatch by M (what w4a8_gemm does)                          */
+    W4A8_PATH_SPLITK = 1,    /* weight-streaming split-K kernel (M <= 64 only)               */
+    W4A8_PATH_TCGEN05 = 2    /* TMA + tcgen05.mma kind::i8 + TMEM kernel (any M)             */
+} w4a8_path;
+
+const char* w4a8_status_string(w4a8_status s);
+
+/* Size in bytes of the packed weight blob for an [N,K] layer; 0 for an unsupported shape. */
+size_t w4a8_packed_bytes(int N, int K, int group);
+
+/*
+ * Size in bytes of the scratch workspace w4a8_gemm needs for any M <= M_max on this
+ * layer shape (split-K slices, per-tile arrival counters, one status word); 0 for an
+ * unsupported shape.  The first W4A8_WORKSPACE_HEADER_BYTES bytes must be zero before the
+ * first call (w4a8_workspace_init does that) and are left zero by every call, so one
+ * workspace can serve any number of calls that do not overlap on the GPU.
+ */
+#define W4A8_WORKSPACE_HEADER_BYTES 4096
+size_t w4a8_workspace_bytes(int M_max, int N, int K, int group);
+w4a8_status w4a8_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Offline weight packing (Sec. 3.4: weights are quantised to 4 bits once, offline).  A pure
+ * re-ordering of codes, scales and zero points into the layout the GEMM kernels stream.
+ *   qw      [N,K] row-major, one code per byte (only the low 4 bits are used)
+ *   scales  [K/group, N] fp16 bit patterns
+ *   zeros   [K/group, N] one zero point per byte (low 4 bits)
+ *   packed_out  w4a8_packed_bytes(N,K,group) bytes, 128-byte aligned
+ */
+w4a8_status w4a8_pack_weights(const uint8_t* qw, const uint16_t* scales, const uint8_t* zeros,
+                              int N, int K, int group, void* packed_out, void* stream);
+
+/* Inverse of w4a8_pack_weights (layout round-trip checks).  Any output pointer may be NULL. */
+w4a8_status w4a8_unpack_weights(const void* packed, int N, int K, int group,
+                                uint8_t* qw_out, uint16_t* scales_out, uint8_t* zeros_out,
+                                void* stream);
+
+/*
+ * Per-token dynamic activation quantisation (Sec. 3.4: "8-bit activations").
+ *   x_bf16  [M,K] row-major, contiguous, 16-byte aligned
+ *   qa      [M,K] int8, 16-byte aligned       sa  [M] fp16 bit patterns
+ *   asum    [M,K/group] int32 sums of qa over each group (zero-point correction term)
+ */
+w4a8_status w4a8_quantize_act(const void* x_bf16, int M, int K, int group,
+                              int8_t* qa, uint16_t* sa, int32_t* asum, void* stream);
+
+/*
+ * The quantised linear itself (Sec. 3.4: INT8 tensor-core matmul on 4-bit weights and
+ * 8-bit activations; Sec. 4: memory-bound for decode-sized M, compute-bound for prefill).
+ *   qa, sa, asum     outputs of w4a8_quantize_act (qa 16-byte aligned)
+ *   packed_w         output of w4a8_pack_weights for the same N, K, group
+ *   y_bf16           [M,N] row-major bf16
+ *   workspace        >= w4a8_workspace_bytes(M,N,K,group) bytes, 256-byte aligned, header zeroed once
+ *   debug_partials   NULL, or [M,K/group,N] int32 that receives D (slower debug mode)
+ * Dispatch: M <= 64 runs the split-K weight-streaming kernel, larger M the tcgen05 kernel.
+ * Results are run-to-run deterministic.
+ */
+w4a8_status w4a8_gemm(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
+                      const void* packed_w, void* y_bf16,
+                      int M, int N, int K, int group,
+                      void* workspace, size_t workspace_bytes,
+                      int32_t* debug_partials, void* stream);
+
+/* w4a8_gemm with the kernel family forced (path-consistency tests, benchmarking). */
+w4a8_status w4a8_gemm_path(w4a8_path path,
+                           const int8_t* qa, const uint16_t* sa, const int32_t* asum,
+                           const void* packed_w, void* y_bf16,
+                           int M, int N, int K, int group,
+                           void* workspace, size_t workspace_bytes,
+                           int32_t* debug_partials, void* stream);
+
+/*
+ * Reads back the workspace status word: synchronises `stream`, returns W4A8_OK or
+ * W4A8_ERR_TIMEOUT (a kernel gave up on a bounded wait; its output is then invalid), and
+ * clears the word.  Host-synchronising: for tests and debugging, not for the hot path.
+ */
+w4a8_status w4a8_check_status(void* workspace, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* W4A8_H_ */

@@ -1,0 +1,178 @@
+"""ctypes binding of libw4a8.so: same names as the C ABI, argument marshalling only.
+
+PyTorch is used for device memory and streams; every step of the path runs in the
+library's CUDA kernels.  There is no CPU or eager fallback: if the shared library is
+missing the first call raises.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libw4a8.so")
+
+GROUP = 128
+OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(8)
+PATH_AUTO, PATH_SPLITK, PATH_TCGEN05 = 0, 1, 2
+WORKSPACE_HEADER_BYTES = 4096
+
+EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w4a8_workspace_init",
+           "w4a8_pack_weights", "w4a8_unpack_weights", "w4a8_quantize_act", "w4a8_gemm", "w4a8_gemm_path",
+           "w4a8_check_status")
+
+_lib = None
+
+
+class W4A8Error(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+def lib():
+    """The loaded shared library; raises if it has not been built (python -m paper_2608_12932_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2608_12932_b200.build`; "
+                               "there is no fallback path")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, ci, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.w4a8_status_string.restype = ctypes.c_char_p
+        L.w4a8_status_string.argtypes = [ci]
+        L.w4a8_packed_bytes.restype = sz
+        L.w4a8_packed_bytes.argtypes = [ci, ci, ci]
+        L.w4a8_workspace_bytes.restype = sz
+        L.w4a8_workspace_bytes.argtypes = [ci, ci, ci, ci]
+        L.w4a8_workspace_init.restype = ci
+        L.w4a8_workspace_init.argtypes = [vp, sz, vp]
+        L.w4a8_pack_weights.restype = ci
+        L.w4a8_pack_weights.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp]
+        L.w4a8_unpack_weights.restype = ci
+        L.w4a8_unpack_weights.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp]
+        L.w4a8_quantize_act.restype = ci
+        L.w4a8_quantize_act.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp]
+        L.w4a8_gemm.restype = ci
+        L.w4a8_gemm.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp, vp]
+        L.w4a8_gemm_path.restype = ci
+        L.w4a8_gemm_path.argtypes = [ci, vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp, vp]
+        L.w4a8_check_status.restype = ci
+        L.w4a8_check_status.argtypes = [vp, vp]
+        _lib = L
+    return _lib
+
+
+def status_string(code):
+    return lib().w4a8_status_string(int(code)).decode()
+
+
+def _check(code, where):
+    if code != OK:
+        raise W4A8Error(code, where)
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _ptr(t):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def _dev(t, dtype, name):
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: need a contiguous CUDA tensor of {dtype}, got {t.dtype} on {t.device}")
+    return t
+
+
+def w4a8_packed_bytes(N, K, group=GROUP):
+    return int(lib().w4a8_packed_bytes(N, K, group))
+
+
+def w4a8_workspace_bytes(M_max, N, K, group=GROUP):
+    return int(lib().w4a8_workspace_bytes(M_max, N, K, group))
+
+
+def new_workspace(M_max, N, K, group=GROUP, device="cuda", stream=None):
+    """Allocates (through torch) and initialises a workspace for w4a8_gemm on this layer shape."""
+    nbytes = w4a8_workspace_bytes(M_max, N, K, group)
+    if nbytes == 0:
+        raise W4A8Error(ERR_SHAPE, "w4a8_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    _check(lib().w4a8_workspace_init(_ptr(ws), nbytes, _stream(stream)), "w4a8_workspace_init")
+    return ws
+
+
+def w4a8_pack_weights(qw, scales, zeros, group=GROUP, out=None, stream=None):
+    """qw uint8 [N,K] codes, scales fp16 [G,N], zeros uint8 [G,N] -> packed uint8 blob (device)."""
+    _dev(qw, torch.uint8, "qw"), _dev(scales, torch.float16, "scales"), _dev(zeros, torch.uint8, "zeros")
+    N, K = qw.shape
+    nbytes = w4a8_packed_bytes(N, K, group)
+    if nbytes == 0 or tuple(scales.shape) != (K // group, N) or tuple(zeros.shape) != (K // group, N):
+        raise W4A8Error(ERR_SHAPE, "w4a8_pack_weights")
+    if out is None:
+        out = torch.empty(nbytes, dtype=torch.uint8, device=qw.device)
+    _check(lib().w4a8_pack_weights(_ptr(qw), _ptr(scales), _ptr(zeros), N, K, group, _ptr(out), _stream(stream)),
+           "w4a8_pack_weights")
+    return out
+
+
+def w4a8_unpack_weights(packed, N, K, group=GROUP, stream=None):
+    _dev(packed, torch.uint8, "packed")
+    G = K // group
+    qw = torch.empty((N, K), dtype=torch.uint8, device=packed.device)
+    scales = torch.empty((G, N), dtype=torch.float16, device=packed.device)
+    zeros = torch.empty((G, N), dtype=torch.uint8, device=packed.device)
+    _check(lib().w4a8_unpack_weights(_ptr(packed), N, K, group, _ptr(qw), _ptr(scales), _ptr(zeros), _stream(stream)),
+           "w4a8_unpack_weights")
+    return qw, scales, zeros
+
+
+def w4a8_quantize_act(x, group=GROUP, out=None, stream=None):
+    """x bf16 [M,K] -> (qa int8 [M,K], sa fp16 [M], asum int32 [M,K/group])."""
+    _dev(x, torch.bfloat16, "x")
+    M, K = x.shape
+    if out is None:
+        qa = torch.empty((M, K), dtype=torch.int8, device=x.device)
+        sa = torch.empty((M,), dtype=torch.float16, device=x.device)
+        asum = torch.empty((M, max(K // group, 0)), dtype=torch.int32, device=x.device)
+    else:
+        qa, sa, asum = out
+    _check(lib().w4a8_quantize_act(_ptr(x), M, K, group, _ptr(qa), _ptr(sa), _ptr(asum), _stream(stream)),
+           "w4a8_quantize_act")
+    return qa, sa, asum
+
+
+def w4a8_gemm(qa, sa, asum, packed_w, N, workspace, group=GROUP, out=None, debug_partials=None,
+              path=PATH_AUTO, stream=None):
+    """y bf16 [M,N] = the W4A8 linear of quantised activations against a packed layer."""
+    _dev(qa, torch.int8, "qa"), _dev(sa, torch.float16, "sa"), _dev(asum, torch.int32, "asum")
+    _dev(packed_w, torch.uint8, "packed_w"), _dev(workspace, torch.uint8, "workspace")
+    M, K = qa.shape
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=qa.device)
+    else:
+        _dev(out, torch.bfloat16, "out")
+    if debug_partials is not None:
+        _dev(debug_partials, torch.int32, "debug_partials")
+    if path == PATH_AUTO:
+        code = lib().w4a8_gemm(_ptr(qa), _ptr(sa), _ptr(asum), _ptr(packed_w), _ptr(out), M, N, K, group,
+                               _ptr(workspace), workspace.numel(), _ptr(debug_partials), _stream(stream))
+    else:
+        code = lib().w4a8_gemm_path(path, _ptr(qa), _ptr(sa), _ptr(asum), _ptr(packed_w), _ptr(out), M, N, K, group,
+                                    _ptr(workspace), workspace.numel(), _ptr(debug_partials), _stream(stream))
+    _check(code, "w4a8_gemm")
+    return out
+
+
+def w4a8_check_status(workspace, stream=None):
+    _check(lib().w4a8_check_status(_ptr(workspace), _stream(stream)), "w4a8_check_status")
+
+
+def w4a8_linear(x, packed_w, N, workspace, group=GROUP, stream=None):
+    """Convenience: quantise activations, then the GEMM (two library calls on one stream)."""
+    qa, sa, asum = w4a8_quantize_act(x, group, stream=stream)
+    return w4a8_gemm(qa, sa, asum, packed_w, N, workspace, group, stream=stream)

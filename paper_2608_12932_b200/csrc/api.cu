@@ -1,0 +1,153 @@
+// extern "C" boundary of libw4a8: argument validation, dispatch by M, status codes.
+// Every step of the path runs in the CUDA kernels; nothing here touches the data.
+#include <cuda_runtime.h>
+#include "w4a8_internal.cuh"
+
+using namespace w4a8;
+
+namespace {
+
+bool shape_ok(int N, int K, int group) {
+    return group == GROUP && N > 0 && K > 0 && N % TILE_N == 0 && K % GROUP == 0 && N / TILE_N <= MAX_N_TILES;
+}
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+w4a8_status arch_check() {
+    static int cached[64] = {0};      // 0 unknown, 1 ok, 2 wrong arch
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return W4A8_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return W4A8_ERR_CUDA;
+    if (!cached[dev]) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return W4A8_ERR_CUDA;
+        cached[dev] = (major == 10) ? 1 : 2;
+    }
+    return cached[dev] == 1 ? W4A8_OK : W4A8_ERR_ARCH;
+}
+
+size_t slices_bytes(int M, int N, int K) {
+    const int m = M < SPLITK_MAX_M ? M : SPLITK_MAX_M;
+    const int S = splitk_num_slices(m, N, K);
+    return S > 1 ? (size_t)S * m * N * sizeof(float) : 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* w4a8_status_string(w4a8_status s) {
+    switch (s) {
+        case W4A8_OK: return "ok";
+        case W4A8_ERR_NULL: return "null pointer";
+        case W4A8_ERR_SHAPE: return "unsupported shape (need group == 128, K % 128 == 0, N % 128 == 0, M >= 0)";
+        case W4A8_ERR_ALIGN: return "misaligned pointer";
+        case W4A8_ERR_WORKSPACE: return "workspace too small";
+        case W4A8_ERR_ARCH: return "device is not sm_100";
+        case W4A8_ERR_CUDA: return "CUDA call failed";
+        case W4A8_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+size_t w4a8_packed_bytes(int N, int K, int group) {
+    if (!shape_ok(N, K, group)) return 0;
+    return (size_t)(N / TILE_N) * (K / GROUP) * BLOB_BYTES;
+}
+
+size_t w4a8_workspace_bytes(int M_max, int N, int K, int group) {
+    if (!shape_ok(N, K, group) || M_max < 0) return 0;
+    return WS_HEADER_BYTES + slices_bytes(M_max, N, K);
+}
+
+w4a8_status w4a8_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+    if (!workspace) return W4A8_ERR_NULL;
+    if (workspace_bytes < WS_HEADER_BYTES) return W4A8_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return W4A8_ERR_ALIGN;
+    if (cudaMemsetAsync(workspace, 0, WS_HEADER_BYTES, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return W4A8_ERR_CUDA;
+    return W4A8_OK;
+}
+
+w4a8_status w4a8_pack_weights(const uint8_t* qw, const uint16_t* scales, const uint8_t* zeros,
+                              int N, int K, int group, void* packed_out, void* stream) {
+    if (!shape_ok(N, K, group)) return W4A8_ERR_SHAPE;
+    if (!qw || !scales || !zeros || !packed_out) return W4A8_ERR_NULL;
+    if (!aligned(qw, 8) || !aligned(scales, 2) || !aligned(packed_out, 128)) return W4A8_ERR_ALIGN;
+    w4a8_status a = arch_check();
+    if (a != W4A8_OK) return a;
+    return launch_pack_weights(qw, scales, zeros, N, K, packed_out, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+w4a8_status w4a8_unpack_weights(const void* packed, int N, int K, int group,
+                                uint8_t* qw_out, uint16_t* scales_out, uint8_t* zeros_out, void* stream) {
+    if (!shape_ok(N, K, group)) return W4A8_ERR_SHAPE;
+    if (!packed) return W4A8_ERR_NULL;
+    if (!aligned(packed, 128) || (qw_out && !aligned(qw_out, 8)) || (scales_out && !aligned(scales_out, 2)))
+        return W4A8_ERR_ALIGN;
+    w4a8_status a = arch_check();
+    if (a != W4A8_OK) return a;
+    return launch_unpack_weights(packed, N, K, qw_out, scales_out, zeros_out, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+w4a8_status w4a8_quantize_act(const void* x_bf16, int M, int K, int group,
+                              int8_t* qa, uint16_t* sa, int32_t* asum, void* stream) {
+    if (group != GROUP || K <= 0 || K % GROUP != 0 || M < 0) return W4A8_ERR_SHAPE;
+    if (M == 0) return W4A8_OK;
+    if (!x_bf16 || !qa || !sa || !asum) return W4A8_ERR_NULL;
+    if (!aligned(x_bf16, 16) || !aligned(qa, 16) || !aligned(sa, 2) || !aligned(asum, 4)) return W4A8_ERR_ALIGN;
+    w4a8_status a = arch_check();
+    if (a != W4A8_OK) return a;
+    return launch_quantize_act(x_bf16, M, K, qa, sa, asum, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+w4a8_status w4a8_gemm_path(w4a8_path path,
+                           const int8_t* qa, const uint16_t* sa, const int32_t* asum,
+                           const void* packed_w, void* y_bf16,
+                           int M, int N, int K, int group,
+                           void* workspace, size_t workspace_bytes,
+                           int32_t* debug_partials, void* stream) {
+    if (!shape_ok(N, K, group) || M < 0) return W4A8_ERR_SHAPE;
+    if (path != W4A8_PATH_AUTO && path != W4A8_PATH_SPLITK && path != W4A8_PATH_TCGEN05) return W4A8_ERR_SHAPE;
+    if (path == W4A8_PATH_SPLITK && M > SPLITK_MAX_M) return W4A8_ERR_SHAPE;
+    if (M == 0) return W4A8_OK;
+    if (!qa || !sa || !asum || !packed_w || !y_bf16 || !workspace) return W4A8_ERR_NULL;
+    if (!aligned(qa, 16) || !aligned(sa, 2) || !aligned(asum, 4) || !aligned(packed_w, 128) ||
+        !aligned(y_bf16, 2) || !aligned(workspace, 256) || (debug_partials && !aligned(debug_partials, 4)))
+        return W4A8_ERR_ALIGN;
+    if (workspace_bytes < w4a8_workspace_bytes(M, N, K, group)) return W4A8_ERR_WORKSPACE;
+    w4a8_status a = arch_check();
+    if (a != W4A8_OK) return a;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool small = path == W4A8_PATH_SPLITK || (path == W4A8_PATH_AUTO && M <= SPLITK_MAX_M);
+    cudaError_t e = small
+        ? launch_gemm_splitk(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace, debug_partials, st)
+        : launch_gemm_tcgen05(qa, sa, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
+    return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+w4a8_status w4a8_gemm(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
+                      const void* packed_w, void* y_bf16,
+                      int M, int N, int K, int group,
+                      void* workspace, size_t workspace_bytes,
+                      int32_t* debug_partials, void* stream) {
+    return w4a8_gemm_path(W4A8_PATH_AUTO, qa, sa, asum, packed_w, y_bf16, M, N, K, group,
+                          workspace, workspace_bytes, debug_partials, stream);
+}
+
+w4a8_status w4a8_check_status(void* workspace, void* stream) {
+    if (!workspace) return W4A8_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t word = 0;
+    if (cudaMemcpyAsync(&word, static_cast<uint8_t*>(workspace) + WS_STATUS_OFF, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return W4A8_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return W4A8_ERR_CUDA;
+    if (word == 0) return W4A8_OK;
+    if (cudaMemsetAsync(static_cast<uint8_t*>(workspace) + WS_STATUS_OFF, 0, 4, st) != cudaSuccess) return W4A8_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return W4A8_ERR_CUDA;
+    return word == W4A8_ERR_TIMEOUT ? W4A8_ERR_TIMEOUT : W4A8_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,349 @@
+// Large-M W4A8 GEMM for sm_100a: TMA -> shared memory -> int4->int8 unpack in shared memory
+// -> tcgen05.mma kind::i8 with int32 accumulators in TMEM -> per-group fp32 scaling -> bf16.
+// (Sec. 3.4: "8-bit activations unlock faster INT8 matrix multiplies for the compute-heavy
+// prefill"; Sec. 4: prefill is one long matrix multiplication.)
+//
+// Orientation ("swap-AB"): the 128 output channels of a tile are the MMA's M side (TMEM lanes),
+// the tokens are its N side (TMEM columns).  A drain thread therefore owns ONE output channel:
+// its group scale is a per-thread scalar and the per-group work on the CUDA cores is one
+// int->float convert and one FMA per accumulator element.
+//
+// One pipeline step = one quantisation group = 128 k = four K=32 MMAs; the accumulator must
+// be drained after every group because the scale changes, so TMEM holds two accumulator
+// buffers: the tensor core fills one while the drain warps empty the other.
+//
+// Zero points are subtracted while unpacking (weights become signed, -15..15), so the int32
+// accumulator is directly D = sum (q_w - z) q_a; identical to P - z*sum(q_a), and it moves the
+// correction from the per-(token, channel, group) drain to the per-weight unpack.
+//
+// Warp roles (512 threads, four warpgroups so that setmaxnreg can move registers to the drain):
+//   warp 0       producer: 1-D bulk copy of the packed blob, 2-D TMA load of the activation tile
+//   warp 1       MMA issuer (one thread), owns TMEM allocation
+//   warps 4-7    unpack: raw blob -> signed int8 A tile in the 128-byte-swizzled K-major layout
+//   warps 8-15   drain: tcgen05.ld -> convert -> FMA with the group scale; final bf16 store
+// Every wait is bounded; on expiry the CTA records W4A8_ERR_TIMEOUT, frees TMEM and exits.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include "ptx_sm100.cuh"
+#include "w4a8_internal.cuh"
+
+namespace w4a8 {
+namespace {
+
+constexpr int TC_THREADS = 512;
+constexpr int WARP_PRODUCER = 0, WARP_MMA = 1, WARP_UNPACK0 = 4, WARP_DRAIN0 = 8;
+constexpr int NUM_UNPACK_WARPS = 4, NUM_DRAIN_WARPS = 8;
+constexpr int RAW_STAGES = 4;
+constexpr int RAW_STRIDE = 8576;                 // BLOB_BYTES rounded up to a multiple of 128
+constexpr int A_BYTES = TILE_N * GROUP;          // 16384: 128 rows x 128 B, signed int8
+
+template <int TILE_M>
+struct Cfg {
+    static constexpr int AB_STAGES = (TILE_M == 256) ? 3 : 4;
+    static constexpr int B_BYTES = TILE_M * GROUP;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int RAW_OFF = AB_STAGES * STAGE_BYTES;
+    static constexpr int BAR_OFF = RAW_OFF + RAW_STAGES * RAW_STRIDE;
+    static constexpr int NUM_BARS = 2 * RAW_STAGES + 3 * AB_STAGES + 4 + 1;
+    static constexpr int MISC_OFF = BAR_OFF + NUM_BARS * 8;
+    static constexpr int SA_OFF = MISC_OFF + 16;   // per drain warp: token scales as fp32
+    static constexpr int SMEM_BYTES = SA_OFF + NUM_DRAIN_WARPS * (TILE_M / 2) * 4;
+    static constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;       // slack to align the base to 1024 B
+    static constexpr int TMEM_COLS = 2 * TILE_M;               // two accumulator buffers
+    static constexpr int HALF = TILE_M / 2;                    // columns per drain warp
+    static_assert(TILE_M == 64 || TILE_M == 128 || TILE_M == 256, "token tile");
+    static_assert(SMEM_ALLOC <= 227 * 1024, "shared memory");
+};
+
+__device__ __forceinline__ uint32_t sub_zero4(uint32_t q, uint32_t zz) {
+    // bytes of q in 0..15, bytes of zz = z in 0..15: per-byte q - z as signed int8, no borrow
+    return ((q | 0x80808080u) - zz) ^ 0x80808080u;
+}
+
+template <int TILE_M, bool DEBUG>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* __restrict__ packed,
+                    const uint16_t* __restrict__ sa, __nv_bfloat16* __restrict__ y,
+                    int32_t* __restrict__ debug_partials, uint32_t* __restrict__ status,
+                    int M, int N, int K, int m_tiles, int total_tiles) {
+    using C = Cfg<TILE_M>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+    const int G = K / GROUP;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    auto bar = [&](int i) { return smem_base + C::BAR_OFF + 8 * i; };
+    const int RAW_FULL = 0, RAW_EMPTY = RAW_STAGES, B_FULL = 2 * RAW_STAGES, A_FULL = B_FULL + C::AB_STAGES,
+              AB_EMPTY = A_FULL + C::AB_STAGES, ACC_FULL = AB_EMPTY + C::AB_STAGES, ACC_EMPTY = ACC_FULL + 2,
+              FINAL = ACC_EMPTY + 2;
+    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(smem + C::MISC_OFF);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + C::MISC_OFF + 4);
+
+    if (warp == WARP_MMA) {
+        if (lane == 0) {
+            *abort_flag = 0;
+            for (int i = 0; i < RAW_STAGES; ++i) {
+                ptx::mbar_init(bar(RAW_FULL + i), 1);
+                ptx::mbar_init(bar(RAW_EMPTY + i), NUM_UNPACK_WARPS);
+            }
+            for (int i = 0; i < C::AB_STAGES; ++i) {
+                ptx::mbar_init(bar(B_FULL + i), 1);
+                ptx::mbar_init(bar(A_FULL + i), NUM_UNPACK_WARPS);
+                ptx::mbar_init(bar(AB_EMPTY + i), 1);
+            }
+            for (int i = 0; i < 2; ++i) {
+                ptx::mbar_init(bar(ACC_FULL + i), 1);
+                ptx::mbar_init(bar(ACC_EMPTY + i), NUM_DRAIN_WARPS);
+            }
+            ptx::mbar_init(bar(FINAL), 1);
+            ptx::fence_mbar_init();
+        }
+        __syncwarp();
+        ptx::tmem_alloc(smem_base + C::MISC_OFF, C::TMEM_COLS);
+        ptx::tmem_relinquish();
+    }
+    if (warp == WARP_PRODUCER && lane == 0) ptx::prefetch_tmap(&tmap_qa);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp < 4) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        if (warp == WARP_PRODUCER && lane == 0) {
+            // ---------------------------------------------------------------- producer ----
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int ntile = tile / m_tiles, mtile = tile % m_tiles;
+                const uint8_t* src = packed + (size_t)ntile * G * BLOB_BYTES;
+                for (int g = 0; g < G; ++g, ++it) {
+                    const uint32_t sr = it % RAW_STAGES, pr = (it / RAW_STAGES) & 1;
+                    if (!(ok = ptx::mbar_wait(bar(RAW_EMPTY + sr), pr ^ 1, abort_flag))) break;
+                    ptx::mbar_arrive_expect_tx(bar(RAW_FULL + sr), BLOB_BYTES);
+                    ptx::bulk_g2s(smem_base + C::RAW_OFF + sr * RAW_STRIDE, src + (size_t)g * BLOB_BYTES, BLOB_BYTES,
+                                  bar(RAW_FULL + sr));
+                    const uint32_t sb = it % C::AB_STAGES, pb = (it / C::AB_STAGES) & 1;
+                    if (!(ok = ptx::mbar_wait(bar(AB_EMPTY + sb), pb ^ 1, abort_flag))) break;
+                    ptx::mbar_arrive_expect_tx(bar(B_FULL + sb), C::B_BYTES);
+                    ptx::tma_load_2d(smem_base + sb * C::STAGE_BYTES + A_BYTES, &tmap_qa, g * GROUP, mtile * TILE_M,
+                                     bar(B_FULL + sb));
+                }
+            }
+            if (!ok) {   // let copies already in flight land before shared memory is released
+                const uint64_t t0 = ptx::globaltimer_ns();
+                while (ptx::globaltimer_ns() - t0 < 200000ull) {}
+            }
+        } else if (warp == WARP_MMA && lane == 0) {
+            // ---------------------------------------------------------------- MMA issuer ----
+            constexpr uint32_t idesc = ptx::idesc_i8(TILE_N, TILE_M, true, true);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                for (int g = 0; g < G; ++g, ++it) {
+                    const uint32_t sb = it % C::AB_STAGES, pb = (it / C::AB_STAGES) & 1;
+                    const uint32_t buf = it & 1, pa = (it >> 1) & 1;
+                    if (!(ok = ptx::mbar_wait(bar(ACC_EMPTY + buf), pa ^ 1, abort_flag))) break;
+                    if (!(ok = ptx::mbar_wait(bar(B_FULL + sb), pb, abort_flag))) break;
+                    if (!(ok = ptx::mbar_wait(bar(A_FULL + sb), pb, abort_flag))) break;
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a_addr = smem_base + sb * C::STAGE_BYTES, b_addr = a_addr + A_BYTES;
+                    const uint32_t d_tmem = tmem_base + buf * TILE_M;
+#pragma unroll
+                    for (int kk = 0; kk < GROUP / 32; ++kk)
+                        ptx::mma_i8_ss(d_tmem, ptx::smem_desc_k_sw128(a_addr + kk * 32),
+                                       ptx::smem_desc_k_sw128(b_addr + kk * 32), idesc, kk > 0 ? 1u : 0u);
+                    ptx::tc_commit(bar(AB_EMPTY + sb));     // operands of this stage consumed
+                    ptx::tc_commit(bar(ACC_FULL + buf));    // accumulator of this group complete
+                }
+            }
+            // nothing may still be executing on the tensor core when TMEM is freed
+            ptx::tc_commit(bar(FINAL));
+            ptx::mbar_wait(bar(FINAL), 0, abort_flag);
+        }
+    } else if (warp < WARP_DRAIN0) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+        // -------------------------------------------------------------------- unpack ----
+        const int u = tid - WARP_UNPACK0 * 32;
+        uint32_t it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            for (int g = 0; g < G; ++g, ++it) {
+                const uint32_t sr = it % RAW_STAGES, pr = (it / RAW_STAGES) & 1;
+                const uint32_t sb = it % C::AB_STAGES, pb = (it / C::AB_STAGES) & 1;
+                if (!(ok = ptx::mbar_wait(bar(RAW_FULL + sr), pr, abort_flag))) break;
+                if (!(ok = ptx::mbar_wait(bar(AB_EMPTY + sb), pb ^ 1, abort_flag))) break;
+                const uint8_t* raw = smem + C::RAW_OFF + sr * RAW_STRIDE;
+                uint8_t* a_tile = smem + sb * C::STAGE_BYTES;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int c = u + 128 * i;            // 16-byte chunk of the blob: 32 consecutive k of one row
+                    const int row = c >> 2, j = c & 3;
+                    const uint4 w = *reinterpret_cast<const uint4*>(raw + c * 16);
+                    const uint32_t z = (raw[BLOB_ZERO_OFF + (row >> 1)] >> ((row & 1) * 4)) & 0xFu;
+                    const uint32_t zz = z * 0x01010101u;
+                    uint4 o0, o1;
+                    o0.x = sub_zero4(w.x & 0x0F0F0F0Fu, zz);
+                    o0.y = sub_zero4((w.x >> 4) & 0x0F0F0F0Fu, zz);
+                    o0.z = sub_zero4(w.y & 0x0F0F0F0Fu, zz);
+                    o0.w = sub_zero4((w.y >> 4) & 0x0F0F0F0Fu, zz);
+                    o1.x = sub_zero4(w.z & 0x0F0F0F0Fu, zz);
+                    o1.y = sub_zero4((w.z >> 4) & 0x0F0F0F0Fu, zz);
+                    o1.z = sub_zero4(w.w & 0x0F0F0F0Fu, zz);
+                    o1.w = sub_zero4((w.w >> 4) & 0x0F0F0F0Fu, zz);
+                    // K-major row of 128 B; 16-byte chunk index XOR (row % 8): the 128-byte swizzle
+                    uint8_t* rowp = a_tile + row * 128;
+                    *reinterpret_cast<uint4*>(rowp + (((2 * j) ^ (row & 7)) << 4)) = o0;
+                    *reinterpret_cast<uint4*>(rowp + (((2 * j + 1) ^ (row & 7)) << 4)) = o1;
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    ptx::mbar_arrive(bar(A_FULL + sb));
+                    ptx::mbar_arrive(bar(RAW_EMPTY + sr));
+                }
+            }
+        }
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 192;");
+        // --------------------------------------------------------------------- drain ----
+        const int q = warp & 3, h = (warp - WARP_DRAIN0) >> 2;
+        const int n_local = q * 32 + lane;
+        uint32_t it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            const int ntile = tile / m_tiles, mtile = tile % m_tiles;
+            const int n = ntile * TILE_N + n_local;
+            const int m_base = mtile * TILE_M + h * C::HALF;
+            const uint8_t* sw_ptr = packed + (size_t)ntile * G * BLOB_BYTES + BLOB_SCALE_OFF + 2 * n_local;
+            float facc[C::HALF];
+#pragma unroll
+            for (int i = 0; i < C::HALF; ++i) facc[i] = 0.0f;
+            // this warp's token scales, widened once per tile (rows past M get 0 and are never stored)
+            float* sa_w = reinterpret_cast<float*>(smem + C::SA_OFF) + (warp - WARP_DRAIN0) * C::HALF;
+            __syncwarp();
+            for (int i = lane; i < C::HALF; i += 32)
+                sa_w[i] = (m_base + i < M) ? __half2float(__ushort_as_half(__ldg(sa + m_base + i))) : 0.0f;
+            __syncwarp();
+            uint16_t sw_bits = __ldg(reinterpret_cast<const uint16_t*>(sw_ptr));
+            for (int g = 0; g < G; ++g, ++it) {
+                const uint32_t buf = it & 1, pa = (it >> 1) & 1;
+                const float sw = __half2float(__ushort_as_half(sw_bits));
+                if (g + 1 < G) sw_bits = __ldg(reinterpret_cast<const uint16_t*>(sw_ptr + (size_t)(g + 1) * BLOB_BYTES));
+                if (!(ok = ptx::mbar_wait(bar(ACC_FULL + buf), pa, abort_flag))) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * TILE_M + h * C::HALF;
+#pragma unroll
+                for (int ch = 0; ch < C::HALF / 32; ++ch) {
+                    uint32_t v[32];
+                    ptx::tmem_ld_32x32(taddr + ch * 32, v);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        facc[ch * 32 + i] = fmaf(sw, (float)(int)v[i], facc[ch * 32 + i]);
+                        if (DEBUG) {
+                            const int m = m_base + ch * 32 + i;
+                            if (m < M) debug_partials[((size_t)m * G + g) * N + n] = (int)v[i];
+                        }
+                    }
+                }
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar(ACC_EMPTY + buf));
+            }
+            if (!ok) break;
+#pragma unroll
+            for (int i = 0; i < C::HALF; ++i) {   // fully unrolled: facc must stay in registers
+                const int m = m_base + i;
+                if (m < M) y[(size_t)m * N + n] = __float2bfloat16_rn(facc[i] * sa_w[i]);
+            }
+        }
+    }
+
+    if (*abort_flag && lane == 0) atomicExch(status, (uint32_t)W4A8_ERR_TIMEOUT);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == WARP_MMA) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+template <int TILE_M, bool DEBUG>
+cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed, void* y, int M, int N, int K,
+                        void* workspace, int32_t* debug_partials, cudaStream_t stream) {
+    using C = Cfg<TILE_M>;
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return cudaErrorNotSupported;
+    CUtensorMap tmap;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)K};
+    const cuuint32_t box[2] = {(cuuint32_t)GROUP, (cuuint32_t)TILE_M};
+    const cuuint32_t estr[2] = {1, 1};
+    if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(qa), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    static int sm_count[64] = {0};
+    static bool attr_done[64] = {false};
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!sm_count[dev]) {
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        sm_count[dev] = sms;
+    }
+    sms = sm_count[dev];
+    if (!attr_done[dev]) {
+        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<TILE_M, DEBUG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 C::SMEM_ALLOC);
+        if (e != cudaSuccess) return e;
+        attr_done[dev] = true;
+    }
+    const int m_tiles = (M + TILE_M - 1) / TILE_M;
+    const int total = m_tiles * (N / TILE_N);
+    const int grid = total < sms ? total : sms;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    gemm_tcgen05_kernel<TILE_M, DEBUG><<<grid, TC_THREADS, C::SMEM_ALLOC, stream>>>(
+        tmap, static_cast<const uint8_t*>(packed), sa, static_cast<__nv_bfloat16*>(y), debug_partials,
+        reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF), M, N, K, m_tiles, total);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
+                                int M, int N, int K, void* workspace, int32_t* debug_partials,
+                                cudaStream_t stream) {
+    if (debug_partials) {
+        if (M <= 64) return launch_tile<64, true>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+        if (M <= 128) return launch_tile<128, true>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+        return launch_tile<256, true>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+    }
+    if (M <= 64) return launch_tile<64, false>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+    if (M <= 128) return launch_tile<128, false>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+    return launch_tile<256, false>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+}
+
+}  // namespace w4a8

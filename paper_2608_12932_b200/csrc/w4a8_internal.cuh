@@ -1,0 +1,54 @@
+// Internal declarations shared by the translation units of libw4a8: packed layout
+// constants, the workspace layout, kernel launchers.  Not part of the public ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "w4a8.h"
+
+namespace w4a8 {
+
+// ---- packed weight layout -----------------------------------------------------------------
+// The [N,K] layer is cut into blobs of 128 output channels x one group of 128 k.  Blob
+// (ntile, g) sits at byte offset (ntile * G + g) * BLOB_BYTES and holds
+//   [0, 8192)     128 rows x 64 B of nibbles.  Row r, 32-bit word kk (0..15) covers
+//                 k0 = g*128 + 8*kk: byte b of the word has code[k0+b] in its low nibble and
+//                 code[k0+4+b] in its high nibble, so  w & 0x0F0F0F0F  and  (w>>4) & 0x0F0F0F0F
+//                 are four consecutive-k bytes each, and a 16-byte chunk unpacks to 32 consecutive k.
+//   [8192, 8448)  128 fp16 scales, row order
+//   [8448, 8512)  128 zero points, two per byte (row 2i low nibble, row 2i+1 high nibble)
+// A blob is exactly the algorithmic 4.15625 bits per weight: no padding.
+constexpr int TILE_N = 128;
+constexpr int GROUP = 128;
+constexpr int BLOB_NIBBLE_BYTES = TILE_N * GROUP / 2;        // 8192
+constexpr int BLOB_SCALE_OFF = BLOB_NIBBLE_BYTES;             // 8192
+constexpr int BLOB_ZERO_OFF = BLOB_SCALE_OFF + TILE_N * 2;    // 8448
+constexpr int BLOB_BYTES = BLOB_ZERO_OFF + TILE_N / 2;        // 8512
+
+// ---- workspace layout -----------------------------------------------------------------------
+//   [0, 4)                    status word (0 = fine, else a w4a8_status written by a kernel)
+//   [256, 256 + 4*n_tiles)    split-K arrival counters, one per 128-channel tile (zero between calls)
+//   [HEADER, ...)             split-K fp32 slices  [S][M][N]
+constexpr int WS_STATUS_OFF = 0;
+constexpr int WS_COUNTER_OFF = 256;
+constexpr int WS_HEADER_BYTES = W4A8_WORKSPACE_HEADER_BYTES;
+constexpr int MAX_N_TILES = (WS_HEADER_BYTES - WS_COUNTER_OFF) / 4;   // 960 tiles = N up to 122880
+
+// ---- split-K path -----------------------------------------------------------------------------
+constexpr int SPLITK_MAX_M = 64;          // tokens the streaming kernel handles (8 blocks of 8)
+constexpr int SPLITK_MAX_GROUPS = 8;      // groups one CTA keeps in shared memory at once
+int splitk_num_slices(int M, int N, int K);
+
+cudaError_t launch_quantize_act(const void* x, int M, int K, int8_t* qa, uint16_t* sa, int32_t* asum,
+                                cudaStream_t stream);
+cudaError_t launch_pack_weights(const uint8_t* qw, const uint16_t* scales, const uint8_t* zeros,
+                                int N, int K, void* packed, cudaStream_t stream);
+cudaError_t launch_unpack_weights(const void* packed, int N, int K, uint8_t* qw, uint16_t* scales,
+                                  uint8_t* zeros, cudaStream_t stream);
+cudaError_t launch_gemm_splitk(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
+                               void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
+                               cudaStream_t stream);
+cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
+                                int M, int N, int K, void* workspace, int32_t* debug_partials,
+                                cudaStream_t stream);
+
+}  // namespace w4a8

@@ -1,0 +1,88 @@
+"""CPU-side checks of the C-ABI library: it loads without a GPU, exports every symbol the
+public header declares, and its shape/size logic (no kernel launches) behaves as documented."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2608_12932_b200 import binding as B
+from paper_2608_12932_b200 import build as libbuild
+from paper_2608_12932_b200 import workload as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    libbuild.build()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "w4a8.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(w4a8_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    names = declared_functions()
+    assert set(names) == set(B.EXPORTS)
+    lib = ctypes.CDLL(B.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_library_needs_no_driver_to_load():
+    # libcuda is resolved lazily by the static runtime, so loading works on a CPU-only host
+    out = os.popen(f"ldd {B.LIB_PATH}").read()
+    assert "libcuda.so" not in out and "libcudart" not in out
+
+
+def test_size_queries():
+    for (K, N) in wl.LAYERS.values():
+        G = K // 128
+        assert B.w4a8_packed_bytes(N, K) == N * K // 2 + G * N * 5 // 2
+        assert B.w4a8_workspace_bytes(0, N, K) == B.WORKSPACE_HEADER_BYTES
+        w8, w16, w64, w4096 = (B.w4a8_workspace_bytes(m, N, K) for m in (8, 16, 64, 4096))
+        assert B.WORKSPACE_HEADER_BYTES < w8 < w16 < w64 == w4096
+        assert (w8 - B.WORKSPACE_HEADER_BYTES) % (8 * N * 4) == 0
+    assert B.w4a8_packed_bytes(100, 256) == 0
+    assert B.w4a8_packed_bytes(128, 100) == 0
+    assert B.w4a8_packed_bytes(128, 256, 64) == 0
+    assert B.w4a8_workspace_bytes(8, 128, 256, 32) == 0
+    assert B.w4a8_workspace_bytes(-1, 128, 256) == 0
+    assert B.w4a8_packed_bytes(128 * 961, 128) == 0          # more tiles than the workspace header has counters
+
+
+def test_status_strings():
+    seen = {B.status_string(c) for c in range(8)}
+    assert len(seen) == 8 and "ok" in seen
+    assert B.status_string(99) == "unknown status"
+
+
+def test_shape_validation_needs_no_gpu():
+    L = B.lib()
+    # shape errors are reported before any CUDA call
+    assert L.w4a8_quantize_act(None, 4, 200, 128, None, None, None, None) == B.ERR_SHAPE
+    assert L.w4a8_quantize_act(None, -1, 256, 128, None, None, None, None) == B.ERR_SHAPE
+    assert L.w4a8_quantize_act(None, 0, 256, 128, None, None, None, None) == B.OK
+    assert L.w4a8_quantize_act(None, 4, 256, 128, None, None, None, None) == B.ERR_NULL
+    assert L.w4a8_pack_weights(None, None, None, 100, 256, 128, None, None) == B.ERR_SHAPE
+    assert L.w4a8_pack_weights(None, None, None, 128, 256, 128, None, None) == B.ERR_NULL
+    assert L.w4a8_gemm(None, None, None, None, None, 8, 128, 256, 64, None, 0, None, None) == B.ERR_SHAPE
+    assert L.w4a8_gemm(None, None, None, None, None, 0, 128, 256, 128, None, 0, None, None) == B.OK
+    assert L.w4a8_gemm(None, None, None, None, None, 8, 128, 256, 128, None, 0, None, None) == B.ERR_NULL
+    assert L.w4a8_gemm_path(7, None, None, None, None, None, 8, 128, 256, 128, None, 0, None, None) == B.ERR_SHAPE
+    assert L.w4a8_gemm_path(B.PATH_SPLITK, None, None, None, None, None, 65, 128, 256, 128, None, 0, None, None) == B.ERR_SHAPE
+    assert L.w4a8_workspace_init(None, 4096, None) == B.ERR_NULL
+    assert L.w4a8_check_status(None, None) == B.ERR_NULL
+    # alignment is checked before the device is queried
+    assert L.w4a8_quantize_act(ctypes.c_void_p(0x1002), 4, 256, 128, ctypes.c_void_p(0x2000),
+                               ctypes.c_void_p(0x3000), ctypes.c_void_p(0x4000), None) == B.ERR_ALIGN
+
+
+def test_missing_library_fails_loudly(tmp_path, monkeypatch):
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no fallback"):
+        B.lib()
