@@ -73,7 +73,7 @@ def test_quantize_edge_rows():
     x[0] = 0.0
     x[1] = -0.0
     x[2] *= np.float32(2.0 ** 100)          # scale saturates at 65504
-    x[3] *= np.float32(2.0 ** -20)          # scale is an fp16 subnormal
+    x[3] *= np.float32(2.0 ** -12)          # scale is an fp16 subnormal
     x[4] *= np.float32(2.0 ** -40)          # scale underflows to zero
     x[5, :] = 3.96875 / 127                 # every quotient equal
     x[5, 0] = 3.96875
