@@ -1,0 +1,454 @@
+#!/usr/bin/env python
+"""Benchmark of the W4A8 quantized linear (Sec. 3.4) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--no-sweep] [--impl reference]
+
+One "step" is one pass of the whole hot path - w4a8_quantize_act then w4a8_gemm - over one
+batch of the speculative-verify configuration (M = 8 draft tokens, K = 4096, N = 6144;
+Sec. 3.2), with the weights packed once beforehand (they are quantised offline, Sec. 3.4).
+That configuration is memory-bound, so the metric is HBM GB/s: algorithmic bytes of the
+step divided by time.  Successive steps use different packed copies of the layer (more
+than two L2 capacities in total), so weights always come from HBM, as they do in a decoder
+that walks through dozens of distinct layers.  The timed region is one CUDA-graph launch of
+exactly K steps, bracketed by CUDA events, a barrier and a device synchronise.
+
+Printed on one JSON line: the step throughput (`value`), the same measured end to end from
+pinned host buffers through w4a8_linear_host (`e2e`), the roofline of the dominant kernel
+(`roofline`), the CPU oracle timed on this host's cores (`cpu_baseline`), the SM clocks seen
+during the timed region (`clocks`), and - unless --no-sweep - TOPS / GB/s / roofline fraction
+for all four linears of the decoder layer at M = 1...4096 (`sweep`).
+
+Multi-GPU: the path does not shard (one GPU per model replica); with --gpus N every rank
+runs the same replica on its own GPU and the value is the sum over ranks (weak scaling).
+`--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_12932_b200 import workload as wl  # noqa: E402
+
+HEADLINE = "spec_verify"
+METRIC = "w4a8_linear_hbm_gbs"
+NOMINAL_HBM_GBS = 8000.0          # "~8 TB/s"
+NOMINAL_INT8_TOPS = 4500.0        # dense INT8, twice the nominal dense bf16 rate
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+L2_BYTES_ASSUMED = 126 * 2 ** 20
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=FALLBACK_HBM_GBS, bf16_tflops=FALLBACK_BF16_TFLOPS,
+                bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def step_bytes(M, N, K):
+    return wl.algorithmic_bytes_quantize(M, K) + wl.algorithmic_bytes_gemm(M, N, K)
+
+
+# ----------------------------------------------------------------------------- clocks ----
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, f"/tmp/w4a8_bench_clocks_{os.getpid()}.csv"
+
+    def start(self):
+        try:
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=self.out, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return None
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.out.close()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                t = [v.strip() for v in line.split(",")]
+                if len(t) < 7:
+                    continue
+                try:
+                    sm.append(float(t[0])), smax.append(float(t[1]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, t[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+        os.unlink(self.path)
+        if not sm:
+            return None
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------- CPU oracle arm ---
+def time_oracle(case, min_seconds, max_steps=None):
+    """The CPU oracle, as it stands, on the whole headline step; returns (steps, seconds, threads)."""
+    from oracle import cfast
+    cfast.build()
+    cfast.w4a8_linear(case["x"], case["qw"], case["sw"], case["z"], case["group"])     # page in
+    steps, t0 = 0, time.perf_counter()
+    while True:
+        cfast.w4a8_linear(case["x"], case["qw"], case["sw"], case["z"], case["group"])
+        steps += 1
+        el = time.perf_counter() - t0
+        if (max_steps is not None and steps >= max_steps) or (max_steps is None and el >= min_seconds):
+            return steps, el, cfast.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    case = wl.make_config(HEADLINE)
+    M, N, K = case["M"], case["N"], case["K"]
+    time_oracle(case, 0.0, max_steps=max(args.warmup, 1))
+    steps, el, threads = time_oracle(case, 0.0, max_steps=args.steps)
+    gbs = step_bytes(M, N, K) * steps / el / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": steps, "warmup": args.warmup, "ms_per_step": el / steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8 x uint4 -> int32, fp64 scaling", "data": "synthetic",
+        "config": {"workload": f"{HEADLINE}: M={M} K={K} N={N} group=128, quantise + W4A8 linear"},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle",
+                         "sample": f"the whole step, {steps} repetitions"},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------ GPU arm ---
+def to_dev16(torch, a, dtype):
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda().view(dtype)
+
+
+class Timer:
+    def __init__(self, torch):
+        self.torch = torch
+
+    def graph_ms(self, fn, replays=1, warm=3):
+        """Capture fn() into a CUDA graph, replay it; returns best and median ms per replay."""
+        torch = self.torch
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            fn()                                   # eager warm-up (sets function attributes before capture)
+        torch.cuda.current_stream().wait_stream(s)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        for _ in range(warm):
+            g.replay()
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(replays):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            g.replay()
+            e1.record()
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1))
+        return g, times
+
+
+def copies_for(nbytes, l2_bytes):
+    return int(np.ceil(2.0 * l2_bytes / nbytes)) + 1
+
+
+def run_sweep(torch, B, peaks, l2_bytes, timer):
+    """All four linears at every M of the sweep: GEMM alone, rotating cold weight copies."""
+    out = []
+    int8_peak = 2.0 * peaks["bf16_tflops"]
+    for lname, (K, N) in wl.LAYERS.items():
+        case = wl.make_sweep_layer(lname)
+        qw = torch.from_numpy(case["qw"]).cuda()
+        sw = to_dev16(torch, case["sw"], torch.float16)
+        z = torch.from_numpy(case["z"]).cuda()
+        packed0 = B.w4a8_pack_weights(qw, sw, z)
+        ncopies = copies_for(packed0.numel(), l2_bytes)
+        packed = [packed0] + [packed0.clone() for _ in range(ncopies - 1)]
+        del qw, sw, z
+        ws = B.new_workspace(max(wl.SWEEP_M), N, K)
+        x_all = to_dev16(torch, case["x"], torch.bfloat16)
+        for M in wl.SWEEP_M:
+            qa, sa, asum = B.w4a8_quantize_act(x_all[:M].contiguous())
+            y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+            reps = 2 if M >= 1024 else 4
+
+            def body():
+                for _ in range(reps):
+                    for p in packed:
+                        B.w4a8_gemm(qa, sa, asum, p, N, ws, out=y)
+            _, times = timer.graph_ms(body, replays=5, warm=2)
+            B.w4a8_check_status(ws)
+            us = min(times) * 1e3 / (reps * ncopies)
+            ops, nbytes = wl.algorithmic_ops(M, N, K), wl.algorithmic_bytes_gemm(M, N, K)
+            t_c_meas, t_m_meas = ops / (int8_peak * 1e12), nbytes / (peaks["hbm_gbs"] * 1e9)
+            t_c_nom, t_m_nom = ops / (NOMINAL_INT8_TOPS * 1e12), nbytes / (NOMINAL_HBM_GBS * 1e9)
+            out.append({"layer": lname, "M": M, "us": round(us, 2),
+                        "tops": round(ops / us / 1e6, 1), "gbs": round(nbytes / us / 1e3, 1),
+                        "bound": "int8" if t_c_meas > t_m_meas else "hbm",
+                        "frac_measured": round(max(t_c_meas, t_m_meas) * 1e6 / us, 3),
+                        "frac_nominal": round(max(t_c_nom, t_m_nom) * 1e6 / us, 3)})
+        del packed, packed0, x_all
+        torch.cuda.empty_cache()
+    return out
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2608_12932_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    B.lib()
+    peaks = measured_peaks()
+    l2_bytes = torch.cuda.get_device_properties(local).L2_cache_size or L2_BYTES_ASSUMED
+    timer = Timer(torch)
+
+    case = wl.make_config(HEADLINE)
+    M, N, K, g = case["M"], case["N"], case["K"], case["group"]
+    qw = torch.from_numpy(case["qw"]).cuda()
+    sw = to_dev16(torch, case["sw"], torch.float16)
+    z = torch.from_numpy(case["z"]).cuda()
+    packed0 = B.w4a8_pack_weights(qw, sw, z, g)                 # offline, once
+    ncopies = copies_for(packed0.numel(), l2_bytes)
+    packed = [packed0] + [packed0.clone() for _ in range(ncopies - 1)]
+    ws = B.new_workspace(M, N, K, g)
+    x = to_dev16(torch, case["x"], torch.bfloat16)
+    qa = torch.empty((M, K), dtype=torch.int8, device="cuda")
+    sa = torch.empty((M,), dtype=torch.float16, device="cuda")
+    asum = torch.empty((M, K // g), dtype=torch.int32, device="cuda")
+    y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+
+    def step(i):
+        B.w4a8_quantize_act(x, g, out=(qa, sa, asum))
+        B.w4a8_gemm(qa, sa, asum, packed[i % ncopies], N, ws, g, out=y)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- correctness of this very launch configuration against the oracle (outside the timed region)
+    from oracle import cfast
+    from oracle import w4a8_oracle as onp
+    step(0)
+    B.w4a8_check_status(ws)
+    ref = cfast.w4a8_linear(case["x"], case["qw"], case["sw"], case["z"], g)
+    ok, ratio = onp.within_tolerance(y.view(torch.int16).cpu().numpy().view(np.uint16), ref["ref"])
+    parity = {"codes_exact": bool(np.array_equal(qa.cpu().numpy(), ref["qa"])), "bf16_within_tolerance": ok,
+              "worst_err_over_bound": round(ratio, 4)}
+
+    # ---- timed region: W warm-up steps, then exactly K steps in one graph launch
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    g_steps = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_steps):
+        for i in range(args.steps):
+            step(i)
+    g_steps.replay()                     # untimed: graph upload, instruction caches
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(local).uuid).replace("GPU-", ""))
+    barrier()
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    g_steps.replay()
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    # keep the GPU in the same state a little longer so the sampler sees clocks under this load
+    t_end = time.perf_counter() + 0.6
+    while time.perf_counter() < t_end:
+        g_steps.replay()
+        torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    B.w4a8_check_status(ws)
+    if world > 1:
+        t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    sbytes = step_bytes(M, N, K)
+    value = sbytes * args.steps * world / (ms_total * 1e-3) / 1e9
+
+    # ---- roofline of the dominant kernel: the split-K GEMM alone, same rotation, K launches
+    def gemm_only():
+        for i in range(args.steps):
+            B.w4a8_gemm(qa, sa, asum, packed[i % ncopies], N, ws, g, out=y)
+    _, gt = timer.graph_ms(gemm_only, replays=5, warm=2)
+    gemm_us = float(np.median(gt)) * 1e3 / args.steps
+    gbytes = wl.algorithmic_bytes_gemm(M, N, K)
+    achieved = gbytes / gemm_us / 1e3
+
+    def quant_only():
+        for i in range(args.steps):
+            B.w4a8_quantize_act(x, g, out=(qa, sa, asum))
+    _, qt = timer.graph_ms(quant_only, replays=5, warm=2)
+    quant_us = float(np.median(qt)) * 1e3 / args.steps
+
+    # ---- end to end from pinned host buffers through w4a8_linear_host, copies inside the timed region
+    x_host = torch.from_numpy(np.ascontiguousarray(case["x"]).view(np.int16)).view(torch.bfloat16).pin_memory()
+    y_host = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    host = B.HostLinear(M, N, K, packed0, ws, g)
+
+    def e2e_steps():
+        for i in range(args.steps):
+            host.packed_w = packed[i % ncopies]
+            host(x_host, y_host)
+    g_e2e, et = timer.graph_ms(e2e_steps, replays=3, warm=2)
+    barrier()
+    e2e_ms = float(np.median(et))
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = sbytes * args.steps * world / (e2e_ms * 1e-3) / 1e9
+    e2e_ok, _ = onp.within_tolerance(y_host.view(torch.int16).numpy().view(np.uint16), ref["ref"])
+    parity["e2e_within_tolerance"] = e2e_ok
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- CPU oracle on this host's cores, same step (bounded: a few seconds)
+    osteps, oel, threads = time_oracle(case, 3.0)
+    cpu_gbs = sbytes * osteps / oel / 1e9
+
+    sweep = None
+    if not args.no_sweep and world == 1:
+        sweep = run_sweep(torch, B, peaks, l2_bytes, timer)
+
+    line = {
+        "metric": METRIC, "value": round(value, 2), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8 x uint4 -> int32 (fp32 scaling, bf16 out)", "data": "synthetic",
+        "config": {"workload": f"{HEADLINE}: M={M} K={K} N={N} group=128; step = w4a8_quantize_act + w4a8_gemm",
+                   "l2": f"{ncopies} distinct packed weight copies visited in turn ({ncopies * packed0.numel() / 2**20:.0f} MiB "
+                         f"> 2 x L2 of {l2_bytes / 2**20:.0f} MiB); activations stay L2-resident as in a real decoder",
+                   "launch": "one CUDA graph of K steps, CUDA events around the replay",
+                   "parallelism": "replicas only" if world > 1 else "1 GPU"},
+        "e2e": {"value": round(e2e_value, 2), "unit": "GB/s", "h2d_bytes_per_step": M * K * 2,
+                "d2h_bytes_per_step": M * N * 2, "ms_per_step": e2e_ms / args.steps},
+        "gpu_launches": 2 * args.steps,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "gemm_splitk_kernel<1>", "achieved": round(achieved, 1),
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4),
+                     "peak_source": f"of {peaks['source']} (STREAM-style copy, burst)",
+                     "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
+                     "us_per_launch": round(gemm_us, 3), "algorithmic_bytes_per_launch": gbytes,
+                     "traffic": TRAFFIC_BYTES_PER_LAUNCH,
+                     "timing": "K back-to-back launches in one graph, inter-launch gaps included"},
+        "kernels_us": {"w4a8_quantize_act": round(quant_us, 3), "w4a8_gemm": round(gemm_us, 3)},
+        "cpu_baseline": {"value": round(cpu_gbs, 3), "unit": "GB/s", "cores": threads, "kind": "oracle",
+                         "sample": f"the whole step (M={M}, all {N} channels), {osteps} repetitions in {oel:.1f} s"},
+        "parity": parity,
+    }
+    if sweep is not None:
+        line["sweep"] = sweep
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_shape(args):
+    """--shape LAYER:M : quantise + GEMM of one sweep point, launched eagerly `steps` times on cold
+    weight copies (the small case that ncu captures are taken on); prints one JSON line."""
+    import torch
+
+    from paper_2608_12932_b200 import binding as B
+    lname, M = args.shape.split(":")
+    M = int(M)
+    K, N = wl.LAYERS[lname]
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    case = wl.make_layer(K, N, wl.LAYER_SEEDS[lname], M)
+    packed0 = B.w4a8_pack_weights(torch.from_numpy(case["qw"]).cuda(), to_dev16(torch, case["sw"], torch.float16),
+                                  torch.from_numpy(case["z"]).cuda())
+    l2_bytes = torch.cuda.get_device_properties(torch.cuda.current_device()).L2_cache_size or L2_BYTES_ASSUMED
+    ncopies = copies_for(packed0.numel(), l2_bytes)
+    packed = [packed0] + [packed0.clone() for _ in range(ncopies - 1)]
+    ws = B.new_workspace(M, N, K)
+    x = to_dev16(torch, case["x"], torch.bfloat16)
+    y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    times = []
+    for i in range(args.warmup + args.steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        qa, sa, asum = B.w4a8_quantize_act(x)
+        e0.record()
+        B.w4a8_gemm(qa, sa, asum, packed[i % ncopies], N, ws, out=y)
+        e1.record()
+        e1.synchronize()
+        if i >= args.warmup:
+            times.append(e0.elapsed_time(e1) * 1e3)
+    B.w4a8_check_status(ws)
+    us = float(np.median(times))
+    print(json.dumps({"shape": args.shape, "M": M, "N": N, "K": K, "gemm_us_eager_median": round(us, 2),
+                      "tops": round(wl.algorithmic_ops(M, N, K) / us / 1e6, 1),
+                      "gbs": round(wl.algorithmic_bytes_gemm(M, N, K) / us / 1e3, 1), "launches": args.steps}))
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one split-K GEMM launch at the headline shape,
+# from the ncu capture summarised under profiles/ (None until a capture exists)
+TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=int(os.environ.get("WORLD_SIZE", "1")))
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--shape", default=None, help="LAYER:M, e.g. gate_up:1024 - run only that GEMM (profiling aid)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.shape:
+        run_shape(args)
+    elif args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -122,6 +122,22 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
                            int32_t* debug_partials, void* stream);
 
 /*
+ * The whole path for callers whose activations and results live in HOST memory (Sec. 3.5: a
+ * pipeline stage is one graph launch fed from the host): enqueues, on `stream`, the copy of
+ * x to the device, w4a8_quantize_act, w4a8_gemm, and the copy of y back to the host.
+ *   x_host_bf16  HOST [M,K] bf16 (pinned memory makes the copies asynchronous)
+ *   y_host_bf16  HOST [M,N] bf16, valid once `stream` has been synchronised by the caller
+ *   x_dev, qa, sa, asum, y_dev   DEVICE staging buffers owned by the caller, sized and aligned
+ *                as for w4a8_quantize_act / w4a8_gemm ([M,K] bf16, [M,K] int8, [M] fp16,
+ *                [M,K/group] int32, [M,N] bf16)
+ * Same shape rules and status codes as w4a8_gemm.
+ */
+w4a8_status w4a8_linear_host(const void* x_host_bf16, void* y_host_bf16,
+                             int M, int N, int K, int group, const void* packed_w,
+                             void* x_dev, int8_t* qa, uint16_t* sa, int32_t* asum, void* y_dev,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Reads back the workspace status word: synchronises `stream`, returns W4A8_OK or
  * W4A8_ERR_TIMEOUT (a kernel gave up on a bounded wait; its output is then invalid), and
  * clears the word.  Host-synchronising: for tests and debugging, not for the hot path.

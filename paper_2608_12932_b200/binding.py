@@ -19,7 +19,7 @@ WORKSPACE_HEADER_BYTES = 4096
 
 EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w4a8_workspace_init",
            "w4a8_pack_weights", "w4a8_unpack_weights", "w4a8_quantize_act", "w4a8_gemm", "w4a8_gemm_path",
-           "w4a8_check_status")
+           "w4a8_linear_host", "w4a8_check_status")
 
 _lib = None
 
@@ -57,6 +57,8 @@ def lib():
         L.w4a8_gemm.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp, vp]
         L.w4a8_gemm_path.restype = ci
         L.w4a8_gemm_path.argtypes = [ci, vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp, vp]
+        L.w4a8_linear_host.restype = ci
+        L.w4a8_linear_host.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.w4a8_check_status.restype = ci
         L.w4a8_check_status.argtypes = [vp, vp]
         _lib = L
@@ -170,6 +172,31 @@ def w4a8_gemm(qa, sa, asum, packed_w, N, workspace, group=GROUP, out=None, debug
 
 def w4a8_check_status(workspace, stream=None):
     _check(lib().w4a8_check_status(_ptr(workspace), _stream(stream)), "w4a8_check_status")
+
+
+class HostLinear:
+    """Device staging buffers for w4a8_linear_host on one layer shape (allocated once, through torch)."""
+
+    def __init__(self, M, N, K, packed_w, workspace, group=GROUP, device="cuda"):
+        self.M, self.N, self.K, self.group = M, N, K, group
+        self.packed_w, self.workspace = packed_w, workspace
+        self.x_dev = torch.empty((M, K), dtype=torch.bfloat16, device=device)
+        self.qa = torch.empty((M, K), dtype=torch.int8, device=device)
+        self.sa = torch.empty((M,), dtype=torch.float16, device=device)
+        self.asum = torch.empty((M, K // group), dtype=torch.int32, device=device)
+        self.y_dev = torch.empty((M, N), dtype=torch.bfloat16, device=device)
+
+    def __call__(self, x_host, y_host, stream=None):
+        """x_host, y_host: CPU bf16 tensors (pinned for asynchronous copies); enqueues the whole path."""
+        if x_host.is_cuda or y_host.is_cuda or x_host.dtype != torch.bfloat16 or y_host.dtype != torch.bfloat16:
+            raise TypeError("w4a8_linear_host takes CPU bf16 tensors")
+        if tuple(x_host.shape) != (self.M, self.K) or tuple(y_host.shape) != (self.M, self.N):
+            raise W4A8Error(ERR_SHAPE, "w4a8_linear_host")
+        _check(lib().w4a8_linear_host(_ptr(x_host), _ptr(y_host), self.M, self.N, self.K, self.group,
+                                      _ptr(self.packed_w), _ptr(self.x_dev), _ptr(self.qa), _ptr(self.sa),
+                                      _ptr(self.asum), _ptr(self.y_dev), _ptr(self.workspace),
+                                      self.workspace.numel(), _stream(stream)), "w4a8_linear_host")
+        return y_host
 
 
 def w4a8_linear(x, packed_w, N, workspace, group=GROUP, stream=None):
