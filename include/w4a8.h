@@ -138,6 +138,31 @@ w4a8_status w4a8_linear_host(const void* x_host_bf16, void* y_host_bf16,
                              void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * w4a8_gemm for callers that cannot allocate device memory.  (The paper has no counterpart to
+ * this entry point; it exists for deployment reasons only.)  Some hosts of this library may
+ * not call cudaMalloc at all: a control loop with a hard deadline cannot afford the
+ * device-wide synchronisation and unbounded latency an allocation may cost, and a component
+ * running inside another runtime's pre-partitioned memory pool has no allocator of its own to
+ * obtain a workspace from.  For them the split-K scratch (slices, arrival counters, status word)
+ * is a fixed array of W4A8_STATIC_SCRATCH_BYTES bytes inside the library image; every GPU that
+ * loads the library holds that much memory until the process exits.
+ *   - Same inputs, output and shape rules as w4a8_gemm, restricted to the split-K path: M <= 64.
+ *   - A shape whose scratch need (4096 + S*M*N*4 bytes, S = number of K slices the library
+ *     picks for N and K) exceeds W4A8_STATIC_SCRATCH_BYTES is refused with W4A8_ERR_WORKSPACE;
+ *     nothing is enqueued.
+ *   - Calls no cudaMalloc, cudaFree or other allocating routine.  The first call on each device
+ *     performs a one-time set-up (it looks up the array's device address and sets a kernel
+ *     attribute); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array, and each call zeroes the array's header on
+ *     `stream` before its kernel: two calls that overlap on the GPU (different streams) race.
+ *     Serialise them on one stream.
+ */
+#define W4A8_STATIC_SCRATCH_BYTES (4096 + 4 * 1024 * 1024)
+w4a8_status w4a8_gemm_static_scratch(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
+                                     const void* packed_w, void* y_bf16,
+                                     int M, int N, int K, int group, void* stream);
+
+/*
  * Reads back the workspace status word: synchronises `stream`, returns W4A8_OK or
  * W4A8_ERR_TIMEOUT (a kernel gave up on a bounded wait; its output is then invalid), and
  * clears the word.  Host-synchronising: for tests and debugging, not for the hot path.

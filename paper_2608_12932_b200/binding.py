@@ -19,7 +19,7 @@ WORKSPACE_HEADER_BYTES = 4096
 
 EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w4a8_workspace_init",
            "w4a8_pack_weights", "w4a8_unpack_weights", "w4a8_quantize_act", "w4a8_gemm", "w4a8_gemm_path",
-           "w4a8_linear_host", "w4a8_check_status")
+           "w4a8_linear_host", "w4a8_gemm_static_scratch", "w4a8_check_status")
 
 _lib = None
 
@@ -59,6 +59,8 @@ def lib():
         L.w4a8_gemm_path.argtypes = [ci, vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp, vp]
         L.w4a8_linear_host.restype = ci
         L.w4a8_linear_host.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.w4a8_gemm_static_scratch.restype = ci
+        L.w4a8_gemm_static_scratch.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp]
         L.w4a8_check_status.restype = ci
         L.w4a8_check_status.argtypes = [vp, vp]
         _lib = L
@@ -167,6 +169,25 @@ def w4a8_gemm(qa, sa, asum, packed_w, N, workspace, group=GROUP, out=None, debug
         code = lib().w4a8_gemm_path(path, _ptr(qa), _ptr(sa), _ptr(asum), _ptr(packed_w), _ptr(out), M, N, K, group,
                                     _ptr(workspace), workspace.numel(), _ptr(debug_partials), _stream(stream))
     _check(code, "w4a8_gemm")
+    return out
+
+
+STATIC_SCRATCH_BYTES = 4096 + 4 * 1024 * 1024
+
+
+def w4a8_gemm_static_scratch(qa, sa, asum, packed_w, N, group=GROUP, out=None, stream=None):
+    """w4a8_gemm without a workspace argument, for callers that cannot allocate device memory:
+    the split-K scratch is a fixed array inside the library (M <= 64, scratch need at most
+    STATIC_SCRATCH_BYTES).  `out` must be given by such callers; it is allocated here otherwise."""
+    _dev(qa, torch.int8, "qa"), _dev(sa, torch.float16, "sa"), _dev(asum, torch.int32, "asum")
+    _dev(packed_w, torch.uint8, "packed_w")
+    M, K = qa.shape
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=qa.device)
+    else:
+        _dev(out, torch.bfloat16, "out")
+    _check(lib().w4a8_gemm_static_scratch(_ptr(qa), _ptr(sa), _ptr(asum), _ptr(packed_w), _ptr(out), M, N, K, group,
+                                          _stream(stream)), "w4a8_gemm_static_scratch")
     return out
 
 

@@ -251,3 +251,59 @@ cudaError_t launch_gemm_splitk(const int8_t* qa, const uint16_t* sa, const int32
 }
 
 }  // namespace w4a8
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant of the split-K GEMM (declared in w4a8.h as w4a8_gemm_static_scratch).
+// The split-K slices, arrival counters and status word live in a fixed array that is part of the
+// library image on every GPU that loads it, instead of a caller-provided workspace.
+namespace w4a8 {
+namespace {
+static __device__ __align__(256) unsigned char g_static_scratch[W4A8_STATIC_SCRATCH_BYTES];
+
+// Device address of g_static_scratch on the current device (0 on failure).  In host code the
+// array's name is only a handle for the runtime, not an address a kernel could use, so the
+// address is looked up once per device with that device current, and cached.
+void* static_scratch_ptr(int dev, cudaError_t* err) {
+    static void* cached[64] = {nullptr};
+    if (!cached[dev]) {
+        void* p = nullptr;
+        *err = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (*err != cudaSuccess) return nullptr;
+        cached[dev] = p;
+    }
+    *err = cudaSuccess;
+    return cached[dev];
+}
+}  // namespace
+}  // namespace w4a8
+
+extern "C" w4a8_status w4a8_gemm_static_scratch(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
+                                                const void* packed_w, void* y_bf16,
+                                                int M, int N, int K, int group, void* stream) {
+    using namespace w4a8;
+    if (group != GROUP || N <= 0 || K <= 0 || N % TILE_N != 0 || K % GROUP != 0 || N / TILE_N > MAX_N_TILES || M < 0)
+        return W4A8_ERR_SHAPE;
+    if (M > SPLITK_MAX_M) return W4A8_ERR_SHAPE;
+    if (M == 0) return W4A8_OK;
+    if (!qa || !sa || !asum || !packed_w || !y_bf16) return W4A8_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(qa) & 15) || (reinterpret_cast<uintptr_t>(sa) & 1) ||
+        (reinterpret_cast<uintptr_t>(asum) & 3) || (reinterpret_cast<uintptr_t>(packed_w) & 127) ||
+        (reinterpret_cast<uintptr_t>(y_bf16) & 1))
+        return W4A8_ERR_ALIGN;
+    const int S = splitk_num_slices(M, N, K);
+    const size_t need = (size_t)WS_HEADER_BYTES + (S > 1 ? (size_t)S * M * N * sizeof(float) : 0);
+    if (need > (size_t)W4A8_STATIC_SCRATCH_BYTES) return W4A8_ERR_WORKSPACE;   // beyond the fixed scratch
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return W4A8_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return W4A8_ERR_CUDA;
+    if (major != 10) return W4A8_ERR_ARCH;
+    cudaError_t e = cudaSuccess;
+    void* scratch = static_scratch_ptr(dev, &e);
+    if (!scratch) return W4A8_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the array keeps whatever the previous call left: the header (status word, arrival counters)
+    // must be zero when the kernel starts
+    if (cudaMemsetAsync(scratch, 0, WS_HEADER_BYTES, st) != cudaSuccess) return W4A8_ERR_CUDA;
+    e = launch_gemm_splitk(qa, sa, asum, packed_w, y_bf16, M, N, K, scratch, nullptr, st);
+    return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
