@@ -17,7 +17,8 @@
  * M tokens, K in-features, N out-features, G = K / group.  y = x W^T with W stored [N,K].
  *
  * Conventions for every entry point
- *   - All data pointers are DEVICE pointers owned by the caller.  Inputs are only read,
+ *   - All data pointers are DEVICE pointers owned by the caller (w4a8_linear_host marks its two
+ *     HOST arguments).  Inputs are only read,
  *     outputs are fully overwritten.  Nothing is allocated or freed by the library.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Work is
  *     enqueued on it; the host is never synchronised (w4a8_check_status excepted).
@@ -51,8 +52,11 @@ typedef enum {
 /* Which GEMM kernel family w4a8_gemm_path runs. */
 typedef enum {
     W4A8_PATH_AUTO = 0,      /* dispatch by M (what w4a8_gemm does)                          */
-    W4A8_PATH_SPLITK = 1,    /* weight-streaming split-K kernel (M <= 64 only)               */
-    W4A8_PATH_TCGEN05 = 2    /* TMA + tcgen05.mma kind::i8 + TMEM kernel (any M)             */
+    W4A8_PATH_SPLITK = 1,    /* weight-streaming split-K kernel, slices reduced inside a
+                                thread-block cluster through distributed shared memory (M <= 64) */
+    W4A8_PATH_TCGEN05 = 2,   /* TMA + tcgen05.mma kind::i8 + TMEM kernel (any M)             */
+    W4A8_PATH_SPLITK_WORKSPACE = 3  /* split-K kernel that reduces its slices through the global
+                                workspace (M <= 64); what w4a8_gemm_static_scratch runs        */
 } w4a8_path;
 
 const char* w4a8_status_string(w4a8_status s);
@@ -105,7 +109,10 @@ w4a8_status w4a8_quantize_act(const void* x_bf16, int M, int K, int group,
  *   workspace        >= w4a8_workspace_bytes(M,N,K,group) bytes, 256-byte aligned, header zeroed once
  *   debug_partials   NULL, or [M,K/group,N] int32 that receives D (slower debug mode)
  * Dispatch: M <= 64 runs the split-K weight-streaming kernel, larger M the tcgen05 kernel.
- * Results are run-to-run deterministic.
+ * Results are run-to-run deterministic.  The kernels are launched with programmatic stream
+ * serialisation: when consecutive library calls share a stream, a kernel may start (and prefetch
+ * weights) before its predecessor has finished, and waits on the device before it reads any
+ * activation or writes any output.
  */
 w4a8_status w4a8_gemm(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
                       const void* packed_w, void* y_bf16,

@@ -110,8 +110,10 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
                            void* workspace, size_t workspace_bytes,
                            int32_t* debug_partials, void* stream) {
     if (!shape_ok(N, K, group) || M < 0) return W4A8_ERR_SHAPE;
-    if (path != W4A8_PATH_AUTO && path != W4A8_PATH_SPLITK && path != W4A8_PATH_TCGEN05) return W4A8_ERR_SHAPE;
-    if (path == W4A8_PATH_SPLITK && M > SPLITK_MAX_M) return W4A8_ERR_SHAPE;
+    if (path != W4A8_PATH_AUTO && path != W4A8_PATH_SPLITK && path != W4A8_PATH_TCGEN05 &&
+        path != W4A8_PATH_SPLITK_WORKSPACE)
+        return W4A8_ERR_SHAPE;
+    if ((path == W4A8_PATH_SPLITK || path == W4A8_PATH_SPLITK_WORKSPACE) && M > SPLITK_MAX_M) return W4A8_ERR_SHAPE;
     if (M == 0) return W4A8_OK;
     if (!qa || !sa || !asum || !packed_w || !y_bf16 || !workspace) return W4A8_ERR_NULL;
     if (!aligned(qa, 16) || !aligned(sa, 2) || !aligned(asum, 4) || !aligned(packed_w, 128) ||
@@ -121,10 +123,13 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
     w4a8_status a = arch_check();
     if (a != W4A8_OK) return a;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool small = path == W4A8_PATH_SPLITK || (path == W4A8_PATH_AUTO && M <= SPLITK_MAX_M);
-    cudaError_t e = small
-        ? launch_gemm_splitk(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace, debug_partials, st)
-        : launch_gemm_tcgen05(qa, sa, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
+    cudaError_t e;
+    if (path == W4A8_PATH_SPLITK_WORKSPACE)
+        e = launch_gemm_splitk(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
+    else if (path == W4A8_PATH_SPLITK || (path == W4A8_PATH_AUTO && M <= SPLITK_MAX_M))
+        e = launch_gemm_cluster(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
+    else
+        e = launch_gemm_tcgen05(qa, sa, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
     return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
 

@@ -1,0 +1,302 @@
+// Small-M W4A8 GEMM, cluster variant: the K slices of one 128-channel tile form a thread-block
+// cluster and are reduced through distributed shared memory, so the kernel needs no global
+// scratch, no atomics and no memory fence.  (Sec. 3.2: a draft block is 8 tokens; Sec. 4: decode is
+// bound by the weight bytes the GPU must load - this kernel streams them once at HBM width.)
+//
+//  * grid = tiles x S, cluster = the S slices of a tile (S <= 8).  A CTA walks its consecutive
+//    groups through a ring of R stages; one stage = one packed blob (1-D bulk copy, 8512 B) plus
+//    the matching 128-byte-wide activation tile (2-D TMA, 128-byte swizzle, rows >= M read as 0).
+//  * a producer warp issues the copies; the weight copies of the first R stages are issued before
+//    griddepcontrol.wait, so under programmatic dependent launch the weight stream of this
+//    kernel overlaps the tail of the previous kernel in the stream.
+//  * eight consumer warps: mma.sync m16n8k32 (u8 x s8 -> s32), weights as the 16-row operand;
+//    D = P - z * sum(q_a) with the group sums from the quantise kernel; fp32 group scales.
+//  * reduction: every CTA leaves its fp32 partial tile in its own shared memory; after a cluster
+//    barrier CTA r sums, for its 1/S share of the tile, the S partials in rank order (fixed
+//    order: deterministic), applies the token scale and stores bf16; a second cluster barrier
+//    keeps every CTA's shared memory alive until its peers have read it.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include "ptx_sm100.cuh"
+#include "w4a8_internal.cuh"
+
+namespace w4a8 {
+namespace {
+
+constexpr int CL_CONSUMER_WARPS = 8;
+constexpr int CL_THREADS = (CL_CONSUMER_WARPS + 1) * 32;   // + one producer warp
+constexpr int CL_MAX_STAGES = 6;
+constexpr int CL_BLOB_STRIDE = 8704;                       // BLOB_BYTES rounded up to a multiple of 128
+constexpr int CL_RED_STRIDE = 132;                         // floats per token row of the partial tile (conflict-free)
+constexpr int CL_MAX_S = 8;
+
+struct ClLayout {
+    int act_off, blob_off, bar_off, asum_off, red_off, misc_off, total;
+};
+__host__ __device__ inline ClLayout cl_layout(int mb, int stages, int ng_max) {
+    ClLayout L;
+    L.act_off = 0;                                            // stages x (8*mb rows x 128 B), 1024-aligned
+    L.blob_off = L.act_off + stages * 1024 * mb;
+    L.bar_off = L.blob_off + stages * CL_BLOB_STRIDE;
+    L.asum_off = L.bar_off + 2 * CL_MAX_STAGES * 8;
+    L.red_off = (L.asum_off + 8 * mb * ng_max * 4 + 15) & ~15;
+    L.misc_off = L.red_off + 8 * mb * CL_RED_STRIDE * 4;
+    L.total = L.misc_off + 16;
+    return L;
+}
+
+__device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int MB>
+__global__ void __launch_bounds__(CL_THREADS)
+gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t* __restrict__ sa,
+                    const int32_t* __restrict__ asum, const uint8_t* __restrict__ packed,
+                    __nv_bfloat16* __restrict__ y, int M, int N, int K, int S, int ng_max, int stages,
+                    uint32_t* __restrict__ status, int32_t* __restrict__ debug_partials) {
+    ptx::pdl_launch_dependents();
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+    const ClLayout L = cl_layout(MB, stages, ng_max);
+    constexpr int MP = 8 * MB;
+    constexpr uint32_t ACT_BYTES = MP * GROUP;
+
+    const int G = K / GROUP;
+    const int ntile = blockIdx.x / S;
+    const int slice = (int)ptx::cluster_ctarank();             // == blockIdx.x % S
+    const int g0 = (int)(((long long)slice * G) / S), g1 = (int)(((long long)(slice + 1) * G) / S);
+    const int ng = g1 - g0;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    auto full_bar = [&](int s) { return smem_base + L.bar_off + 8 * s; };
+    auto empty_bar = [&](int s) { return smem_base + L.bar_off + 8 * (CL_MAX_STAGES + s); };
+    int32_t* asum_s = reinterpret_cast<int32_t*>(smem + L.asum_off);
+    float* red = reinterpret_cast<float*>(smem + L.red_off);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L.misc_off);
+    const uint8_t* src = packed + ((size_t)ntile * G + g0) * BLOB_BYTES;
+
+    if (warp == CL_CONSUMER_WARPS && lane == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < stages; ++s) {
+            ptx::mbar_init(full_bar(s), 1);
+            ptx::mbar_init(empty_bar(s), CL_CONSUMER_WARPS);
+        }
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tmap_qa);
+        // weights do not depend on the previous kernel: start their stream at once
+        const int first = ng < stages ? ng : stages;
+        for (int gi = 0; gi < first; ++gi) {
+            ptx::mbar_expect_tx(full_bar(gi), BLOB_BYTES);
+            ptx::bulk_g2s(smem_base + L.blob_off + gi * CL_BLOB_STRIDE, src + (size_t)gi * BLOB_BYTES, BLOB_BYTES,
+                          full_bar(gi));
+        }
+    }
+    __syncthreads();
+    // Activations, their scales and group sums come from the previous kernel.  They are read
+    // only after this wait and only through L2 (TMA, ld.global.cg): an L1 line filled by an
+    // older grid that shared this SM could otherwise be stale.
+    ptx::pdl_wait();
+
+    float facc[MB][4];
+#pragma unroll
+    for (int mb = 0; mb < MB; ++mb) facc[mb][0] = facc[mb][1] = facc[mb][2] = facc[mb][3] = 0.0f;
+    const int r = lane >> 2, j = lane & 3;
+    const int row_lo = (warp & 7) * 16 + r, row_hi = row_lo + 8;
+
+    if (warp == CL_CONSUMER_WARPS) {
+        // ------------------------------------------------------------------ producer ----
+        if (lane == 0) {
+            bool ok = true;
+            for (int gi = 0; gi < ng && ok; ++gi) {
+                const int s = gi % stages;
+                if (gi >= stages) {
+                    ok = ptx::mbar_wait(empty_bar(s), ((gi / stages) - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    ptx::mbar_arrive_expect_tx(full_bar(s), BLOB_BYTES + ACT_BYTES);
+                    ptx::bulk_g2s(smem_base + L.blob_off + s * CL_BLOB_STRIDE, src + (size_t)gi * BLOB_BYTES,
+                                  BLOB_BYTES, full_bar(s));
+                } else {
+                    ptx::mbar_arrive_expect_tx(full_bar(s), ACT_BYTES);    // blob bytes were announced above
+                }
+                ptx::tma_load_2d(smem_base + L.act_off + s * 1024 * MB, &tmap_qa, (g0 + gi) * GROUP, 0, full_bar(s));
+            }
+        }
+    } else {
+        // ----------------------------------------------------------------- consumers ----
+        for (int i = tid; i < MP * ng; i += CL_CONSUMER_WARPS * 32) {
+            const int m = i / ng, gi = i % ng;
+            asum_s[m * ng_max + gi] = (m < M) ? __ldcg(asum + (size_t)m * G + g0 + gi) : 0;
+        }
+        ptx::named_bar_sync(1, CL_CONSUMER_WARPS * 32);
+        bool ok = true;
+        for (int gi = 0; gi < ng; ++gi) {
+            const int s = gi % stages;
+            ok = ptx::mbar_wait(full_bar(s), (gi / stages) & 1, abort_flag);
+            if (!ok) break;
+            const uint8_t* blob = smem + L.blob_off + s * CL_BLOB_STRIDE;
+            const uint8_t* act = smem + L.act_off + s * 1024 * MB;
+            const uint4 wa = *reinterpret_cast<const uint4*>(blob + row_lo * 64 + j * 16);
+            const uint4 wb = *reinterpret_cast<const uint4*>(blob + row_hi * 64 + j * 16);
+            const uint32_t wlo[4] = {wa.x, wa.y, wa.z, wa.w}, whi[4] = {wb.x, wb.y, wb.z, wb.w};
+            uint32_t a[4][4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                a[q][0] = wlo[q] & 0x0F0F0F0Fu;            // row_lo, k = 32j + 8q + 0..3
+                a[q][1] = whi[q] & 0x0F0F0F0Fu;            // row_hi, same k
+                a[q][2] = (wlo[q] >> 4) & 0x0F0F0F0Fu;     // row_lo, k = 32j + 8q + 4..7
+                a[q][3] = (whi[q] >> 4) & 0x0F0F0F0Fu;     // row_hi
+            }
+            const uint16_t* sc = reinterpret_cast<const uint16_t*>(blob + BLOB_SCALE_OFF);
+            const float s_lo = __half2float(__ushort_as_half(sc[row_lo]));
+            const float s_hi = __half2float(__ushort_as_half(sc[row_hi]));
+            const int z_lo = (blob[BLOB_ZERO_OFF + (row_lo >> 1)] >> ((row_lo & 1) * 4)) & 0xF;
+            const int z_hi = (blob[BLOB_ZERO_OFF + (row_hi >> 1)] >> ((row_hi & 1) * 4)) & 0xF;
+#pragma unroll
+            for (int mb = 0; mb < MB; ++mb) {
+                // token row 8*mb + r of the stage: 128 B, 16-byte chunks XOR-swizzled by the row index
+                const uint8_t* arow = act + mb * 1024 + r * 128;
+                const uint4 b0 = *reinterpret_cast<const uint4*>(arow + (((2 * j) ^ r) << 4));
+                const uint4 b1 = *reinterpret_cast<const uint4*>(arow + (((2 * j + 1) ^ r) << 4));
+                const uint32_t bq[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                int c[4] = {0, 0, 0, 0};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) mma_u8s8(c, a[q][0], a[q][1], a[q][2], a[q][3], bq[2 * q], bq[2 * q + 1]);
+                const int m0 = 8 * mb + 2 * j;
+                const int A0 = asum_s[m0 * ng_max + gi], A1 = asum_s[(m0 + 1) * ng_max + gi];
+                const int d0 = c[0] - z_lo * A0, d1 = c[1] - z_lo * A1;
+                const int d2 = c[2] - z_hi * A0, d3 = c[3] - z_hi * A1;
+                facc[mb][0] = fmaf(s_lo, (float)d0, facc[mb][0]);
+                facc[mb][1] = fmaf(s_lo, (float)d1, facc[mb][1]);
+                facc[mb][2] = fmaf(s_hi, (float)d2, facc[mb][2]);
+                facc[mb][3] = fmaf(s_hi, (float)d3, facc[mb][3]);
+                if (debug_partials) {
+                    const size_t n_lo = (size_t)ntile * TILE_N + row_lo, n_hi = n_lo + 8;
+                    const int g = g0 + gi;
+                    if (m0 < M) {
+                        debug_partials[((size_t)m0 * G + g) * N + n_lo] = d0;
+                        debug_partials[((size_t)m0 * G + g) * N + n_hi] = d2;
+                    }
+                    if (m0 + 1 < M) {
+                        debug_partials[((size_t)(m0 + 1) * G + g) * N + n_lo] = d1;
+                        debug_partials[((size_t)(m0 + 1) * G + g) * N + n_hi] = d3;
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(empty_bar(s));
+        }
+        if (!ok) {
+            // copies of stages not yet consumed may still be in flight: give them a bounded time to land
+            for (int gi = 0; gi < ng && gi < stages; ++gi)
+                for (int spin = 0; spin < (1 << 16) && !ptx::mbar_try_wait(full_bar(gi % stages), 0); ++spin) {}
+        }
+        // partial tile of this slice -> own shared memory
+#pragma unroll
+        for (int mb = 0; mb < MB; ++mb) {
+            const int m0 = 8 * mb + 2 * j;
+            red[m0 * CL_RED_STRIDE + row_lo] = facc[mb][0];
+            red[(m0 + 1) * CL_RED_STRIDE + row_lo] = facc[mb][1];
+            red[m0 * CL_RED_STRIDE + row_hi] = facc[mb][2];
+            red[(m0 + 1) * CL_RED_STRIDE + row_hi] = facc[mb][3];
+        }
+    }
+    if (*abort_flag && lane == 0) atomicExch(status, (uint32_t)W4A8_ERR_TIMEOUT);
+
+    __syncwarp();
+    ptx::cluster_sync();
+    {
+        const int T = M * TILE_N;
+        const int lo = (int)(((long long)slice * T) / S), hi = (int)(((long long)(slice + 1) * T) / S);
+        const uint32_t red_addr = smem_base + L.red_off;
+        uint32_t peer[CL_MAX_S];
+#pragma unroll
+        for (int s = 0; s < CL_MAX_S; ++s) peer[s] = ptx::map_to_cta(red_addr, (uint32_t)(s < S ? s : 0));
+        for (int idx = lo + tid; idx < hi; idx += CL_THREADS) {
+            const int m = idx / TILE_N, nn = idx % TILE_N;
+            const uint32_t off = (uint32_t)(m * CL_RED_STRIDE + nn) * 4u;
+            float p[CL_MAX_S];
+#pragma unroll
+            for (int s = 0; s < CL_MAX_S; ++s) p[s] = (s < S) ? ptx::ld_dsmem_f32(peer[s] + off) : 0.0f;
+            float acc = 0.0f;
+#pragma unroll
+            for (int s = 0; s < CL_MAX_S; ++s) acc += p[s];            // rank order: deterministic
+            const float t = __half2float(__ushort_as_half(__ldcg(sa + m)));
+            y[(size_t)m * N + (size_t)ntile * TILE_N + nn] = __float2bfloat16_rn(acc * t);
+        }
+    }
+    __syncwarp();
+    ptx::cluster_sync();
+}
+
+template <int MB>
+cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed, void* y,
+                      int M, int N, int K, int S, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
+    const int G = K / GROUP;
+    const int ng_max = (G + S - 1) / S;
+    const int stages = ng_max < CL_MAX_STAGES ? ng_max : CL_MAX_STAGES;
+    const ClLayout L = cl_layout(MB, stages, ng_max);
+    const size_t smem = (size_t)L.total + 1024;
+    if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    static bool attr_done[64] = {false};
+    if (!attr_done[dev]) {
+        e = cudaFuncSetAttribute(gemm_cluster_kernel<MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_done[dev] = true;
+    }
+    CUtensorMap tmap;
+    e = make_qa_tensor_map(&tmap, qa, M, K, 8 * MB);
+    if (e != cudaSuccess) return e;
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((N / TILE_N) * S), 1, 1);
+    cfg.blockDim = dim3(CL_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attrs[2];
+    attrs[0].id = cudaLaunchAttributeClusterDimension;
+    attrs[0].val.clusterDim.x = (unsigned)S;
+    attrs[0].val.clusterDim.y = 1;
+    attrs[0].val.clusterDim.z = 1;
+    attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attrs;
+    cfg.numAttrs = 2;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    return cudaLaunchKernelEx(&cfg, gemm_cluster_kernel<MB>, tmap, sa, asum, static_cast<const uint8_t*>(packed),
+                              static_cast<__nv_bfloat16*>(y), M, N, K, S, ng_max, stages,
+                              reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF), debug_partials);
+}
+}  // namespace
+
+// Slices per tile for the cluster kernel: about two CTAs per SM, at most 8 (portable cluster size),
+// never more than the number of groups.
+int cluster_num_slices(int N, int K) {
+    const int G = K / GROUP, tiles = N / TILE_N;
+    int s = (2 * 148 + tiles / 2) / tiles;
+    if (s > CL_MAX_S) s = CL_MAX_S;
+    if (s > G) s = G;
+    if (s < 1) s = 1;
+    return s;
+}
+
+cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
+                                void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
+                                cudaStream_t stream) {
+    const int S = cluster_num_slices(N, K);
+    if (M <= 8) return launch_mb<1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+    if (M <= 16) return launch_mb<2>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+    if (M <= 32) return launch_mb<4>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+    return launch_mb<8>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+}
+
+}  // namespace w4a8

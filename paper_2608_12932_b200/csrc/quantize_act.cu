@@ -9,6 +9,7 @@
 // break exact ties).  Group sums of the codes (the zero-point correction term) come from
 // a 16-lane segmented shuffle: 16 chunks of 8 = one group of 128.
 #include <cuda_fp16.h>
+#include "ptx_sm100.cuh"
 #include "w4a8_internal.cuh"
 
 namespace w4a8 {
@@ -49,6 +50,10 @@ __device__ __forceinline__ uint2 quant8(const uint4& v, float s, int& sum) {
 __global__ void __launch_bounds__(QA_THREADS)
 quantize_act_kernel(const uint4* __restrict__ x, int K, uint2* __restrict__ qa,
                     uint16_t* __restrict__ sa, int32_t* __restrict__ asum) {
+    // Under programmatic dependent launch this grid may start while its predecessor still runs:
+    // let the next grid start as early, and touch no memory before the predecessor is complete.
+    ptx::pdl_launch_dependents();
+    ptx::pdl_wait();
     const int m = blockIdx.x;
     const int chunks = K >> 3;                    // 16-byte chunks per row; a multiple of 16
     const int G = K >> 7;
@@ -62,12 +67,12 @@ quantize_act_kernel(const uint4* __restrict__ x, int K, uint2* __restrict__ qa,
     for (int i = 0; i < QA_CACHE; ++i) {
         int c = tid + i * QA_THREADS;
         if (c < chunks) {
-            cache[i] = __ldg(xr + c);
+            cache[i] = __ldcg(xr + c);
             run = absmax_bits_bf16x8(cache[i], run);
         }
     }
     for (int c = tid + QA_CACHE * QA_THREADS; c < chunks; c += QA_THREADS)
-        run = absmax_bits_bf16x8(__ldg(xr + c), run);
+        run = absmax_bits_bf16x8(__ldcg(xr + c), run);
 
     uint32_t mx = max(run & 0xFFFFu, run >> 16);
     mx = __reduce_max_sync(0xFFFFFFFFu, mx);
@@ -102,16 +107,24 @@ quantize_act_kernel(const uint4* __restrict__ x, int K, uint2* __restrict__ qa,
         int c = tid + i * QA_THREADS;
         if (c < chunks) emit(c, cache[i]);
     }
-    for (int c = tid + QA_CACHE * QA_THREADS; c < chunks; c += QA_THREADS) emit(c, __ldg(xr + c));
+    for (int c = tid + QA_CACHE * QA_THREADS; c < chunks; c += QA_THREADS) emit(c, __ldcg(xr + c));
 }
 
 }  // namespace
 
 cudaError_t launch_quantize_act(const void* x, int M, int K, int8_t* qa, uint16_t* sa, int32_t* asum,
                                 cudaStream_t stream) {
-    quantize_act_kernel<<<M, QA_THREADS, 0, stream>>>(reinterpret_cast<const uint4*>(x), K,
-                                                      reinterpret_cast<uint2*>(qa), sa, asum);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)M, 1, 1);
+    cfg.blockDim = dim3(QA_THREADS, 1, 1);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, quantize_act_kernel, reinterpret_cast<const uint4*>(x), K,
+                              reinterpret_cast<uint2*>(qa), sa, asum);
 }
 
 }  // namespace w4a8

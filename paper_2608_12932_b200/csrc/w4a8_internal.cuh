@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of libw4a8: packed layout
 // constants, the workspace layout, kernel launchers.  Not part of the public ABI.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include "w4a8.h"
@@ -38,6 +39,7 @@ constexpr int SPLITK_MAX_M = 64;          // tokens the streaming kernel handles
 constexpr int SPLITK_MAX_GROUPS = 8;      // groups one CTA keeps in shared memory at once
 int splitk_num_slices(int M, int N, int K);
 
+cudaError_t make_qa_tensor_map(CUtensorMap* out, const int8_t* qa, int M, int K, int box_rows);
 cudaError_t launch_quantize_act(const void* x, int M, int K, int8_t* qa, uint16_t* sa, int32_t* asum,
                                 cudaStream_t stream);
 cudaError_t launch_pack_weights(const uint8_t* qw, const uint16_t* scales, const uint8_t* zeros,
@@ -47,6 +49,10 @@ cudaError_t launch_unpack_weights(const void* packed, int N, int K, uint8_t* qw,
 cudaError_t launch_gemm_splitk(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
                                void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
                                cudaStream_t stream);
+int cluster_num_slices(int N, int K);
+cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
+                                void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
+                                cudaStream_t stream);
 cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
                                 int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream);

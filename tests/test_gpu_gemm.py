@@ -17,7 +17,8 @@ from tests.gpu_util import DeviceLayer, bits, t_u16
 
 pytestmark = pytest.mark.gpu
 
-PATHS = {"splitk": B.PATH_SPLITK, "tcgen05": B.PATH_TCGEN05, "auto": B.PATH_AUTO}
+PATHS = {"splitk": B.PATH_SPLITK, "splitk_ws": B.PATH_SPLITK_WORKSPACE, "tcgen05": B.PATH_TCGEN05,
+         "auto": B.PATH_AUTO}
 
 
 def check_case(case, layer, M, path, debug=True, rows=None):
@@ -39,7 +40,7 @@ def check_case(case, layer, M, path, debug=True, rows=None):
 
 
 # ------------------------------------------------------------------ tiny configuration ---
-@pytest.mark.parametrize("path", ["splitk", "tcgen05", "auto"])
+@pytest.mark.parametrize("path", ["splitk", "splitk_ws", "tcgen05", "auto"])
 def test_tiny_config(path):
     case = wl.make_config("tiny")
     layer = DeviceLayer(case, 16)
@@ -49,7 +50,7 @@ def test_tiny_config(path):
     assert np.array_equal(D, rn["D"])
 
 
-@pytest.mark.parametrize("path", ["splitk", "tcgen05"])
+@pytest.mark.parametrize("path", ["splitk", "splitk_ws", "tcgen05"])
 def test_worked_example_on_gpu(golden, path):
     """The hand-worked example embedded in a 128x128 layer (group 128): same D and y."""
     g = golden("worked_example_w4a8.txt")
@@ -83,10 +84,11 @@ def mid_case():
     return case, DeviceLayer(case, 600)
 
 
+@pytest.mark.parametrize("path", ["splitk", "splitk_ws"])
 @pytest.mark.parametrize("M", [1, 3, 8, 9, 16, 17, 32, 33, 63, 64])
-def test_splitk_token_counts(mid_case, M):
+def test_splitk_token_counts(mid_case, M, path):
     case, layer = mid_case
-    check_case(case, layer, M, "splitk")
+    check_case(case, layer, M, path)
 
 
 @pytest.mark.parametrize("M", [1, 16, 64, 65, 128, 129, 255, 256, 257, 300, 520, 600])
@@ -106,7 +108,19 @@ def test_long_k_many_slices():
     layer = DeviceLayer(case, 70)
     for M in (5, 16, 40):
         check_case(case, layer, M, "splitk")
+        check_case(case, layer, M, "splitk_ws")
     check_case(case, layer, 70, "tcgen05")
+
+
+def test_ring_reuse_many_groups_per_cta():
+    """Wide layer, few slices: each CTA walks more groups than its ring has stages."""
+    case = wl.make_layer(4096, 4096, 34, 24)         # 32 tiles -> 8 slices of 4 groups; and
+    layer = DeviceLayer(case, 24)
+    check_case(case, layer, 24, "splitk")
+    case = wl.make_layer(2048, 24576, 35, 8)         # 192 tiles -> 2 slices of 8 groups > 6 stages
+    layer = DeviceLayer(case, 8)
+    check_case(case, layer, 8, "splitk")
+    check_case(case, layer, 5, "splitk", debug=False)
 
 
 def test_persistent_tiles_more_than_sms():
@@ -118,7 +132,7 @@ def test_persistent_tiles_more_than_sms():
 
 
 # -------------------------------------------------------- invariants on the device -------
-@pytest.mark.parametrize("path,M", [("splitk", 8), ("tcgen05", 130)])
+@pytest.mark.parametrize("path,M", [("splitk", 8), ("splitk_ws", 8), ("splitk", 40), ("tcgen05", 130)])
 def test_zero_point_invariant_and_determinism(mid_case, path, M):
     case, layer = mid_case
     c2 = dict(case)
@@ -140,7 +154,8 @@ def test_both_paths_give_identical_partials(mid_case):
     qa, sa, asum = layer.quantize(case["x"][:M])
     y1, D1 = layer.gemm(qa, sa, asum, path=B.PATH_SPLITK, debug=True)
     y2, D2 = layer.gemm(qa, sa, asum, path=B.PATH_TCGEN05, debug=True)
-    assert np.array_equal(D1, D2)
+    y4, D4 = layer.gemm(qa, sa, asum, path=B.PATH_SPLITK_WORKSPACE, debug=True)
+    assert np.array_equal(D1, D2) and np.array_equal(D1, D4)
     # row independence: row 5 of the M = 48 call equals the M = 1 call on that row
     y3, D3 = layer.gemm(qa[5:6].contiguous(), sa[5:6].contiguous(), asum[5:6].contiguous(), path=B.PATH_SPLITK, debug=True)
     assert np.array_equal(D3[0], D1[5])

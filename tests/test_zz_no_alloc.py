@@ -25,7 +25,8 @@ def test_static_scratch_matches_workspace_entry_point_twice():
     layer = DeviceLayer(case, 16)
     for call, M in enumerate((8, 16)):          # two calls in a row, different token counts
         qa, sa, asum = layer.quantize(case["x"][:M])
-        want, _ = layer.gemm(qa, sa, asum, path=B.PATH_SPLITK)
+        want, _ = layer.gemm(qa, sa, asum, path=B.PATH_SPLITK_WORKSPACE)   # the same kernel, caller's workspace
+        auto, _ = layer.gemm(qa, sa, asum)                                  # what w4a8_gemm picks by itself
         y = torch.full((M, layer.N), float("nan"), dtype=torch.bfloat16, device="cuda")
         B.w4a8_gemm_static_scratch(qa, sa, asum, layer.packed, layer.N, out=y)
         torch.cuda.synchronize()
@@ -34,13 +35,15 @@ def test_static_scratch_matches_workspace_entry_point_twice():
         ok, ratio = onp.within_tolerance(got, onp.bf16_bits_to_f64(want))
         assert ok, f"call {call}: worst |err|/bound = {ratio}"
         assert np.array_equal(got, want), f"call {call}: same kernel, same inputs, different bits"
+        ok, ratio = onp.within_tolerance(got, onp.bf16_bits_to_f64(auto))
+        assert ok, f"call {call} against w4a8_gemm: worst |err|/bound = {ratio}"
 
 
 def test_static_scratch_second_call_same_shape_and_limits():
     case = wl.make_config("tiny")
     layer = DeviceLayer(case, 16)
     qa, sa, asum = layer.quantize(case["x"])
-    want, _ = layer.gemm(qa, sa, asum, path=B.PATH_SPLITK)
+    want, _ = layer.gemm(qa, sa, asum, path=B.PATH_SPLITK_WORKSPACE)
     for _ in range(2):
         y = B.w4a8_gemm_static_scratch(qa, sa, asum, layer.packed, layer.N)
         torch.cuda.synchronize()
