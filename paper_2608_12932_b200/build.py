@@ -38,7 +38,8 @@ def check_ptxas(report):
     for m in re.finditer(r"Compiling entry function '(\S+)' for 'sm_100a'.*?\n.*?(\d+) bytes spill stores.*?\n"
                          r".*?Used (\d+) registers", report, re.S):
         name, spill, regs = m.group(1), int(m.group(2)), int(m.group(3))
-        if spill > 16 and "gemm_" in name:      # a stray register is tolerable, an accumulator array is not
+        limit = 16 if "gemm_tcgen05_kernel" in name else 64
+        if spill > limit and "gemm_" in name:   # a few stray registers are tolerable, an accumulator array is not
             problems.append(f"{name}: {spill} bytes of spill stores")
         if "gemm_tcgen05_kernel" in name and regs != 128:
             problems.append(f"{name}: {regs} registers at launch, setmaxnreg budget assumes 128")

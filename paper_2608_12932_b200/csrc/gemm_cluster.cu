@@ -9,12 +9,19 @@
 //  * a producer warp issues the copies; the weight copies of the first R stages are issued before
 //    griddepcontrol.wait, so under programmatic dependent launch the weight stream of this
 //    kernel overlaps the tail of the previous kernel in the stream.
-//  * eight consumer warps: mma.sync m16n8k32 (u8 x s8 -> s32), weights as the 16-row operand;
-//    D = P - z * sum(q_a) with the group sums from the quantise kernel; fp32 group scales.
-//  * reduction: every CTA leaves its fp32 partial tile in its own shared memory; after a cluster
-//    barrier CTA r sums, for its 1/S share of the tile, the S partials in rank order (fixed
-//    order: deterministic), applies the token scale and stores bf16; a second cluster barrier
-//    keeps every CTA's shared memory alive until its peers have read it.
+//  * sixteen consumer warps in two sets of eight (even / odd groups of the slice; a set's warp owns
+//    16 of the 128 rows): mma.sync m16n8k32 (u8 x s8 -> s32), weights as the 16-row operand;
+//    D = P - z * sum(q_a) with the group sums from the quantise kernel; fp32 group scales; the odd
+//    set's partial sums are added to the even set's through shared memory (fixed order).
+//  * reduction: the tile's M x 128 outputs are split into S contiguous shares, one per CTA of the
+//    cluster.  Every CTA pushes each of its fp32 partials into the owner's shared memory (slot =
+//    pusher's rank) with st.shared::cluster, then one cluster barrier (release/acquire); the owner
+//    sums its S slots in rank order (fixed order: deterministic), applies the token scale and
+//    stores bf16.  After the barrier a CTA reads only its own shared memory, so it may exit freely.
+//  * sizing: the number of slices minimises ceil(CTAs / SMs) * ceil(G / S); a launch that fits in
+//    one wave keeps its CTAs under half an SM's shared memory and prefetches as much of its slice
+//    as fits, so that two consecutive launches can be resident together and the weight stream of
+//    the next overlaps the tail of the current one.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include "ptx_sm100.cuh"
@@ -23,15 +30,15 @@
 namespace w4a8 {
 namespace {
 
-constexpr int CL_CONSUMER_WARPS = 8;
+constexpr int CL_ROW_WARPS = 8;                           // 16 weight rows each: one 128-row blob
+constexpr int CL_CONSUMER_WARPS = 2 * CL_ROW_WARPS;        // two sets: even and odd groups of the slice
 constexpr int CL_THREADS = (CL_CONSUMER_WARPS + 1) * 32;   // + one producer warp
-constexpr int CL_MAX_STAGES = 6;
+constexpr int CL_MAX_STAGES = 12;
 constexpr int CL_BLOB_STRIDE = 8704;                       // BLOB_BYTES rounded up to a multiple of 128
-constexpr int CL_RED_STRIDE = 132;                         // floats per token row of the partial tile (conflict-free)
 constexpr int CL_MAX_S = 8;
 
 struct ClLayout {
-    int act_off, blob_off, bar_off, asum_off, red_off, misc_off, total;
+    int act_off, blob_off, bar_off, asum_off, red_off, set_off, misc_off, total;
 };
 __host__ __device__ inline ClLayout cl_layout(int mb, int stages, int ng_max) {
     ClLayout L;
@@ -40,7 +47,8 @@ __host__ __device__ inline ClLayout cl_layout(int mb, int stages, int ng_max) {
     L.bar_off = L.blob_off + stages * CL_BLOB_STRIDE;
     L.asum_off = L.bar_off + 2 * CL_MAX_STAGES * 8;
     L.red_off = (L.asum_off + 8 * mb * ng_max * 4 + 15) & ~15;
-    L.misc_off = L.red_off + 8 * mb * CL_RED_STRIDE * 4;
+    L.set_off = L.red_off + (8 * mb * TILE_N + CL_MAX_S) * 4;     // S slots x ceil(M*128/S) floats
+    L.misc_off = L.set_off + CL_ROW_WARPS * 32 * 4 * mb * 4;      // odd set's partials: 4*mb floats per thread
     L.total = L.misc_off + 16;
     return L;
 }
@@ -60,6 +68,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
                     __nv_bfloat16* __restrict__ y, int M, int N, int K, int S, int ng_max, int stages,
                     uint32_t* __restrict__ status, int32_t* __restrict__ debug_partials) {
     ptx::pdl_launch_dependents();
+    ptx::cluster_arrive_relaxed();     // "this CTA runs": peers wait for it before they write into it
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
@@ -77,7 +86,6 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
     auto full_bar = [&](int s) { return smem_base + L.bar_off + 8 * s; };
     auto empty_bar = [&](int s) { return smem_base + L.bar_off + 8 * (CL_MAX_STAGES + s); };
     int32_t* asum_s = reinterpret_cast<int32_t*>(smem + L.asum_off);
-    float* red = reinterpret_cast<float*>(smem + L.red_off);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L.misc_off);
     const uint8_t* src = packed + ((size_t)ntile * G + g0) * BLOB_BYTES;
 
@@ -85,7 +93,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
         *abort_flag = 0;
         for (int s = 0; s < stages; ++s) {
             ptx::mbar_init(full_bar(s), 1);
-            ptx::mbar_init(empty_bar(s), CL_CONSUMER_WARPS);
+            ptx::mbar_init(empty_bar(s), CL_ROW_WARPS);              // the one set that consumed the stage
         }
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tmap_qa);
@@ -108,15 +116,18 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
     for (int mb = 0; mb < MB; ++mb) facc[mb][0] = facc[mb][1] = facc[mb][2] = facc[mb][3] = 0.0f;
     const int r = lane >> 2, j = lane & 3;
     const int row_lo = (warp & 7) * 16 + r, row_hi = row_lo + 8;
+    const int set = (warp >> 3) & 1;
 
     if (warp == CL_CONSUMER_WARPS) {
         // ------------------------------------------------------------------ producer ----
         if (lane == 0) {
             bool ok = true;
-            for (int gi = 0; gi < ng && ok; ++gi) {
-                const int s = gi % stages;
+            int s = 0;
+            uint32_t phase = 1;                 // parity of the previous use's "empty" phase
+            for (int gi = 0; gi < ng && ok; ++gi, ++s) {
+                if (s == stages) { s = 0; phase ^= 1; }
                 if (gi >= stages) {
-                    ok = ptx::mbar_wait(empty_bar(s), ((gi / stages) - 1) & 1, abort_flag);
+                    ok = ptx::mbar_wait(empty_bar(s), phase, abort_flag);
                     if (!ok) break;
                     ptx::mbar_arrive_expect_tx(full_bar(s), BLOB_BYTES + ACT_BYTES);
                     ptx::bulk_g2s(smem_base + L.blob_off + s * CL_BLOB_STRIDE, src + (size_t)gi * BLOB_BYTES,
@@ -135,9 +146,11 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
         }
         ptx::named_bar_sync(1, CL_CONSUMER_WARPS * 32);
         bool ok = true;
-        for (int gi = 0; gi < ng; ++gi) {
-            const int s = gi % stages;
-            ok = ptx::mbar_wait(full_bar(s), (gi / stages) & 1, abort_flag);
+        int s = set;
+        uint32_t phase = 0;
+        for (int gi = set; gi < ng; gi += 2, s += 2) {
+            while (s >= stages) { s -= stages; phase ^= 1; }
+            ok = ptx::mbar_wait(full_bar(s), phase, abort_flag);
             if (!ok) break;
             const uint8_t* blob = smem + L.blob_off + s * CL_BLOB_STRIDE;
             const uint8_t* act = smem + L.act_off + s * 1024 * MB;
@@ -164,9 +177,16 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
                 const uint4 b0 = *reinterpret_cast<const uint4*>(arow + (((2 * j) ^ r) << 4));
                 const uint4 b1 = *reinterpret_cast<const uint4*>(arow + (((2 * j + 1) ^ r) << 4));
                 const uint32_t bq[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-                int c[4] = {0, 0, 0, 0};
+                // four independent MMAs (one per k-step) instead of a dependent chain of four
+                int cq[4][4];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) mma_u8s8(c, a[q][0], a[q][1], a[q][2], a[q][3], bq[2 * q], bq[2 * q + 1]);
+                for (int q = 0; q < 4; ++q) {
+                    cq[q][0] = cq[q][1] = cq[q][2] = cq[q][3] = 0;
+                    mma_u8s8(cq[q], a[q][0], a[q][1], a[q][2], a[q][3], bq[2 * q], bq[2 * q + 1]);
+                }
+                int c[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) c[e] = (cq[0][e] + cq[1][e]) + (cq[2][e] + cq[3][e]);
                 const int m0 = 8 * mb + 2 * j;
                 const int A0 = asum_s[m0 * ng_max + gi], A1 = asum_s[(m0 + 1) * ng_max + gi];
                 const int d0 = c[0] - z_lo * A0, d1 = c[1] - z_lo * A1;
@@ -193,45 +213,76 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
         }
         if (!ok) {
             // copies of stages not yet consumed may still be in flight: give them a bounded time to land
-            for (int gi = 0; gi < ng && gi < stages; ++gi)
-                for (int spin = 0; spin < (1 << 16) && !ptx::mbar_try_wait(full_bar(gi % stages), 0); ++spin) {}
+            for (int st = 0; st < stages; ++st)
+                for (int spin = 0; spin < (1 << 16) && !ptx::mbar_try_wait(full_bar(st), 0); ++spin) {}
         }
-        // partial tile of this slice -> own shared memory
+        // odd-group partials join the even-group ones (even + odd: fixed order)
+        float* set_buf = reinterpret_cast<float*>(smem + L.set_off) + ((warp & 7) * 32 + lane) * 4 * MB;
+        if (set == 1) {
 #pragma unroll
-        for (int mb = 0; mb < MB; ++mb) {
-            const int m0 = 8 * mb + 2 * j;
-            red[m0 * CL_RED_STRIDE + row_lo] = facc[mb][0];
-            red[(m0 + 1) * CL_RED_STRIDE + row_lo] = facc[mb][1];
-            red[m0 * CL_RED_STRIDE + row_hi] = facc[mb][2];
-            red[(m0 + 1) * CL_RED_STRIDE + row_hi] = facc[mb][3];
+            for (int mb = 0; mb < MB; ++mb)
+                *reinterpret_cast<float4*>(set_buf + 4 * mb) = make_float4(facc[mb][0], facc[mb][1], facc[mb][2], facc[mb][3]);
+        }
+        ptx::named_bar_sync(1, CL_CONSUMER_WARPS * 32);
+        if (set == 0) {
+#pragma unroll
+            for (int mb = 0; mb < MB; ++mb) {
+                const float4 o = *reinterpret_cast<const float4*>(set_buf + 4 * mb);
+                facc[mb][0] += o.x; facc[mb][1] += o.y; facc[mb][2] += o.z; facc[mb][3] += o.w;
+            }
         }
     }
     if (*abort_flag && lane == 0) atomicExch(status, (uint32_t)W4A8_ERR_TIMEOUT);
 
     __syncwarp();
-    ptx::cluster_sync();
-    {
-        const int T = M * TILE_N;
-        const int lo = (int)(((long long)slice * T) / S), hi = (int)(((long long)(slice + 1) * T) / S);
+    ptx::cluster_wait();       // every CTA of the cluster has started: its shared memory may be written
+    if (warp < CL_ROW_WARPS) {
+        // push this slice's partials to the CTAs that own them: slot `slice` of the owner's buffer
+        const int T = M * TILE_N, chunk = (T + S - 1) / S;
         const uint32_t red_addr = smem_base + L.red_off;
-        uint32_t peer[CL_MAX_S];
+        auto push = [&](int m, int nrow, float v) {
+            if (m < M) {
+                const int idx = m * TILE_N + nrow, owner = idx / chunk;
+                const uint32_t off = (uint32_t)(slice * chunk + idx - owner * chunk) * 4u;
+                ptx::st_dsmem_f32(ptx::map_to_cta(red_addr + off, (uint32_t)owner), v);
+            }
+        };
 #pragma unroll
-        for (int s = 0; s < CL_MAX_S; ++s) peer[s] = ptx::map_to_cta(red_addr, (uint32_t)(s < S ? s : 0));
-        for (int idx = lo + tid; idx < hi; idx += CL_THREADS) {
-            const int m = idx / TILE_N, nn = idx % TILE_N;
-            const uint32_t off = (uint32_t)(m * CL_RED_STRIDE + nn) * 4u;
-            float p[CL_MAX_S];
-#pragma unroll
-            for (int s = 0; s < CL_MAX_S; ++s) p[s] = (s < S) ? ptx::ld_dsmem_f32(peer[s] + off) : 0.0f;
+        for (int mb = 0; mb < MB; ++mb) {
+            const int m0 = 8 * mb + 2 * j;
+            push(m0, row_lo, facc[mb][0]);
+            push(m0 + 1, row_lo, facc[mb][1]);
+            push(m0, row_hi, facc[mb][2]);
+            push(m0 + 1, row_hi, facc[mb][3]);
+        }
+    }
+    __syncwarp();
+    ptx::cluster_sync();       // arrive.release after the pushes, wait.acquire before the sums
+    {
+        const int T = M * TILE_N, chunk = (T + S - 1) / S;
+        const int lo = slice * chunk;
+        const int cnt = (T - lo) < chunk ? (T - lo) : chunk;          // may be <= 0 for the last ranks
+        const float* red = reinterpret_cast<const float*>(smem + L.red_off);
+        for (int i = tid; i < cnt; i += CL_THREADS) {
             float acc = 0.0f;
-#pragma unroll
-            for (int s = 0; s < CL_MAX_S; ++s) acc += p[s];            // rank order: deterministic
+            for (int s = 0; s < S; ++s) acc += red[s * chunk + i];    // rank order: deterministic
+            const int idx = lo + i, m = idx / TILE_N, nn = idx % TILE_N;
             const float t = __half2float(__ushort_as_half(__ldcg(sa + m)));
             y[(size_t)m * N + (size_t)ntile * TILE_N + nn] = __float2bfloat16_rn(acc * t);
         }
     }
-    __syncwarp();
-    ptx::cluster_sync();
+}
+
+int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (!cached[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
 }
 
 template <int MB>
@@ -239,7 +290,24 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
                       int M, int N, int K, int S, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
     const int G = K / GROUP;
     const int ng_max = (G + S - 1) / S;
-    const int stages = ng_max < CL_MAX_STAGES ? ng_max : CL_MAX_STAGES;
+    // shared-memory budget per CTA: a launch of at most one wave leaves room for the next launch's
+    // CTAs on the same SMs; larger launches share the SM between ceil(CTAs/SMs) CTAs of their own
+    const int ctas = (N / TILE_N) * S, sms = sm_count();
+    const int waves = (ctas + sms - 1) / sms;
+    int budget = waves <= 1 ? 110 * 1024 : (220 * 1024) / waves;
+    if (budget < 40 * 1024) budget = 40 * 1024;
+    const int fixed = cl_layout(MB, 0, ng_max).total + 1024;
+    int stages = (budget - fixed) / (CL_BLOB_STRIDE + 1024 * MB);
+    if (stages > CL_MAX_STAGES) stages = CL_MAX_STAGES;
+    if (stages >= ng_max) {
+        stages = ng_max;                       // every stage is used once
+    } else {
+        // Stages are reused.  Even and odd groups go to different warp sets and a parity wait can
+        // only tell consecutive uses of a barrier apart, so each stage must always serve the same
+        // set: the ring length has to be even.
+        stages &= ~1;
+        if (stages < 2) stages = 2;
+    }
     const ClLayout L = cl_layout(MB, stages, ng_max);
     const size_t smem = (size_t)L.total + 1024;
     if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
@@ -262,15 +330,17 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
     cfg.blockDim = dim3(CL_THREADS, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attrs[2];
+    cudaLaunchAttribute attrs[3];
     attrs[0].id = cudaLaunchAttributeClusterDimension;
     attrs[0].val.clusterDim.x = (unsigned)S;
     attrs[0].val.clusterDim.y = 1;
     attrs[0].val.clusterDim.z = 1;
     attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attrs[1].val.programmaticStreamSerializationAllowed = 1;
+    attrs[2].id = cudaLaunchAttributeClusterSchedulingPolicyPreference;     // one CTA per SM before doubling up
+    attrs[2].val.clusterSchedulingPolicyPreference = cudaClusterSchedulingPolicySpread;
     cfg.attrs = attrs;
-    cfg.numAttrs = 2;
+    cfg.numAttrs = 3;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     return cudaLaunchKernelEx(&cfg, gemm_cluster_kernel<MB>, tmap, sa, asum, static_cast<const uint8_t*>(packed),
                               static_cast<__nv_bfloat16*>(y), M, N, K, S, ng_max, stages,
@@ -278,15 +348,18 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
 }
 }  // namespace
 
-// Slices per tile for the cluster kernel: about two CTAs per SM, at most 8 (portable cluster size),
-// never more than the number of groups.
+// Slices per tile for the cluster kernel: the S in 1..8 (portable cluster size; never more than
+// the number of groups) that minimises the longest per-SM chain, ceil(CTAs / SMs) * ceil(G / S);
+// ties go to the smaller S (less to reduce).
 int cluster_num_slices(int N, int K) {
-    const int G = K / GROUP, tiles = N / TILE_N;
-    int s = (2 * 148 + tiles / 2) / tiles;
-    if (s > CL_MAX_S) s = CL_MAX_S;
-    if (s > G) s = G;
-    if (s < 1) s = 1;
-    return s;
+    const int G = K / GROUP, tiles = N / TILE_N, sms = sm_count();
+    int best = 1;
+    long best_cost = -1;
+    for (int s = 1; s <= CL_MAX_S && s <= G; ++s) {
+        const long cost = (long)((tiles * s + sms - 1) / sms) * ((G + s - 1) / s);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+    }
+    return best;
 }
 
 cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,

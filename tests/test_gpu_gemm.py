@@ -247,7 +247,7 @@ def test_decoder_layer_sweep_sampled():
     for lname in wl.LAYERS:
         case = wl.make_sweep_layer(lname)
         layer = DeviceLayer(case, 4096)
-        for M in wl.SWEEP_M:
+        for M in wl.SWEEP_M + (32, 24):          # 32 and 24: the remaining small-M template variants
             x = case["x"][:M]
             qa, sa, asum = layer.quantize(x)
             y, _ = layer.gemm(qa, sa, asum)
