@@ -12,6 +12,13 @@
 // be drained after every group because the scale changes, so TMEM holds two accumulator
 // buffers: the tensor core fills one while the drain warps empty the other.
 //
+// The drain does no int->float conversion: the drain warps re-arm each accumulator buffer with
+// the bit pattern 0x4B400000 (the float 1.5 * 2^23) and every MMA accumulates on top of it.
+// |D| <= 128*15*127 < 2^22, so the int32 sum 0x4B400000 + D read back as a float IS
+// 12582912 + D exactly; one add (minus 12582912) and one FMA with the group scale per element
+// finish the job on the FMA pipe, leaving the ALU pipe to the unpack.  (Packed f32x2
+// arithmetic was measured slower than scalar here.)
+//
 // Zero points are subtracted while unpacking (weights become signed, -15..15), so the int32
 // accumulator is directly D = sum (q_w - z) q_a; identical to P - z*sum(q_a), and it moves the
 // correction from the per-(token, channel, group) drain to the per-weight unpack.
@@ -46,19 +53,22 @@ struct Cfg {
     static constexpr int RAW_OFF = AB_STAGES * STAGE_BYTES;
     static constexpr int BAR_OFF = RAW_OFF + RAW_STAGES * RAW_STRIDE;
     static constexpr int NUM_BARS = 2 * RAW_STAGES + 3 * AB_STAGES + 4 + 1;
-    static constexpr int MISC_OFF = BAR_OFF + NUM_BARS * 8;
+    static constexpr int MISC_OFF = (BAR_OFF + NUM_BARS * 8 + 15) & ~15;        // 16-byte aligned: the staging tile is read with 16-byte loads
     static constexpr int SA_OFF = MISC_OFF + 16;   // per drain warp: token scales as fp32
-    static constexpr int SMEM_BYTES = SA_OFF + NUM_DRAIN_WARPS * (TILE_M / 2) * 4;
+    static constexpr int OUT_OFF = SA_OFF + NUM_DRAIN_WARPS * (TILE_M / 2) * 4;   // per drain warp: 32 tokens x 32 channels bf16
+    static constexpr int SMEM_BYTES = OUT_OFF + NUM_DRAIN_WARPS * 2048;
     static constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;       // slack to align the base to 1024 B
     static constexpr int TMEM_COLS = 2 * TILE_M;               // two accumulator buffers
     static constexpr int HALF = TILE_M / 2;                    // columns per drain warp
     static_assert(TILE_M == 64 || TILE_M == 128 || TILE_M == 256, "token tile");
     static_assert(SMEM_ALLOC <= 227 * 1024, "shared memory");
+    static_assert(OUT_OFF % 16 == 0 && SA_OFF % 16 == 0, "staging alignment");
 };
 
-__device__ __forceinline__ uint32_t sub_zero4(uint32_t q, uint32_t zz) {
-    // bytes of q in 0..15, bytes of zz = z in 0..15: per-byte q - z as signed int8, no borrow
-    return ((q | 0x80808080u) - zz) ^ 0x80808080u;
+__device__ __forceinline__ uint32_t sub_zero4(uint32_t q, uint32_t kz) {
+    // bytes of q in 0..15, bytes of kz = 0x80 - z with z in 0..15: per byte (q + 0x80 - z) ^ 0x80
+    // is q - z as a signed int8; no carry crosses a byte (0x71 <= q + 0x80 - z <= 0x8F)
+    return (q + kz) ^ 0x80808080u;
 }
 
 template <int TILE_M, bool DEBUG>
@@ -111,7 +121,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
     const uint32_t tmem_base = *tmem_holder;
 
     if (warp < 4) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 24;");
         if (warp == WARP_PRODUCER && lane == 0) {
             // ---------------------------------------------------------------- producer ----
             uint32_t it = 0;
@@ -145,7 +155,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 for (int g = 0; g < G; ++g, ++it) {
                     const uint32_t sb = it % C::AB_STAGES, pb = (it / C::AB_STAGES) & 1;
                     const uint32_t buf = it & 1, pa = (it >> 1) & 1;
-                    if (!(ok = ptx::mbar_wait(bar(ACC_EMPTY + buf), pa ^ 1, abort_flag))) break;
+                    if (!(ok = ptx::mbar_wait(bar(ACC_EMPTY + buf), pa, abort_flag))) break;   // re-armed with the bias
                     if (!(ok = ptx::mbar_wait(bar(B_FULL + sb), pb, abort_flag))) break;
                     if (!(ok = ptx::mbar_wait(bar(A_FULL + sb), pb, abort_flag))) break;
                     ptx::tc_fence_after_sync();
@@ -154,7 +164,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
 #pragma unroll
                     for (int kk = 0; kk < GROUP / 32; ++kk)
                         ptx::mma_i8_ss(d_tmem, ptx::smem_desc_k_sw128(a_addr + kk * 32),
-                                       ptx::smem_desc_k_sw128(b_addr + kk * 32), idesc, kk > 0 ? 1u : 0u);
+                                       ptx::smem_desc_k_sw128(b_addr + kk * 32), idesc, 1u);   // on top of the bias
                     ptx::tc_commit(bar(AB_EMPTY + sb));     // operands of this stage consumed
                     ptx::tc_commit(bar(ACC_FULL + buf));    // accumulator of this group complete
                 }
@@ -164,7 +174,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
             ptx::mbar_wait(bar(FINAL), 0, abort_flag);
         }
     } else if (warp < WARP_DRAIN0) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         // -------------------------------------------------------------------- unpack ----
         const int u = tid - WARP_UNPACK0 * 32;
         uint32_t it = 0;
@@ -177,26 +187,29 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 if (!(ok = ptx::mbar_wait(bar(AB_EMPTY + sb), pb ^ 1, abort_flag))) break;
                 const uint8_t* raw = smem + C::RAW_OFF + sr * RAW_STRIDE;
                 uint8_t* a_tile = smem + sb * C::STAGE_BYTES;
+                // one weight row (64 packed bytes -> 128 signed bytes) per thread: its zero point is
+                // fetched once; the four 16-byte chunks are visited in a lane-rotated order so that
+                // the loads of a warp spread over the banks
+                const uint32_t z = (raw[BLOB_ZERO_OFF + (u >> 1)] >> ((u & 1) * 4)) & 0xFu;
+                const uint32_t kz = 0x80808080u - z * 0x01010101u;       // per byte: 0x80 - z, no borrow
+                const uint8_t* rawrow = raw + u * 64;
+                uint8_t* rowp = a_tile + u * 128;
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const int c = u + 128 * i;            // 16-byte chunk of the blob: 32 consecutive k of one row
-                    const int row = c >> 2, j = c & 3;
-                    const uint4 w = *reinterpret_cast<const uint4*>(raw + c * 16);
-                    const uint32_t z = (raw[BLOB_ZERO_OFF + (row >> 1)] >> ((row & 1) * 4)) & 0xFu;
-                    const uint32_t zz = z * 0x01010101u;
+                    const int j = (i + u) & 3;                            // chunk j: k = 32j .. 32j+31
+                    const uint4 w = *reinterpret_cast<const uint4*>(rawrow + j * 16);
                     uint4 o0, o1;
-                    o0.x = sub_zero4(w.x & 0x0F0F0F0Fu, zz);
-                    o0.y = sub_zero4((w.x >> 4) & 0x0F0F0F0Fu, zz);
-                    o0.z = sub_zero4(w.y & 0x0F0F0F0Fu, zz);
-                    o0.w = sub_zero4((w.y >> 4) & 0x0F0F0F0Fu, zz);
-                    o1.x = sub_zero4(w.z & 0x0F0F0F0Fu, zz);
-                    o1.y = sub_zero4((w.z >> 4) & 0x0F0F0F0Fu, zz);
-                    o1.z = sub_zero4(w.w & 0x0F0F0F0Fu, zz);
-                    o1.w = sub_zero4((w.w >> 4) & 0x0F0F0F0Fu, zz);
+                    o0.x = sub_zero4(w.x & 0x0F0F0F0Fu, kz);
+                    o0.y = sub_zero4((w.x >> 4) & 0x0F0F0F0Fu, kz);
+                    o0.z = sub_zero4(w.y & 0x0F0F0F0Fu, kz);
+                    o0.w = sub_zero4((w.y >> 4) & 0x0F0F0F0Fu, kz);
+                    o1.x = sub_zero4(w.z & 0x0F0F0F0Fu, kz);
+                    o1.y = sub_zero4((w.z >> 4) & 0x0F0F0F0Fu, kz);
+                    o1.z = sub_zero4(w.w & 0x0F0F0F0Fu, kz);
+                    o1.w = sub_zero4((w.w >> 4) & 0x0F0F0F0Fu, kz);
                     // K-major row of 128 B; 16-byte chunk index XOR (row % 8): the 128-byte swizzle
-                    uint8_t* rowp = a_tile + row * 128;
-                    *reinterpret_cast<uint4*>(rowp + (((2 * j) ^ (row & 7)) << 4)) = o0;
-                    *reinterpret_cast<uint4*>(rowp + (((2 * j + 1) ^ (row & 7)) << 4)) = o1;
+                    *reinterpret_cast<uint4*>(rowp + (((2 * j) ^ (u & 7)) << 4)) = o0;
+                    *reinterpret_cast<uint4*>(rowp + (((2 * j + 1) ^ (u & 7)) << 4)) = o1;
                 }
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
@@ -207,10 +220,25 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
             }
         }
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 192;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
         // --------------------------------------------------------------------- drain ----
         const int q = warp & 3, h = (warp - WARP_DRAIN0) >> 2;
         const int n_local = q * 32 + lane;
+        constexpr int NCH = C::HALF / 32;                       // 32-column chunks per drain warp
+        constexpr uint32_t ACC_BIAS_BITS = 0x4B400000u;         // 12582912.0f
+        const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + h * C::HALF;
+        // arm both accumulator buffers (this warp's lanes and columns) before the first MMA
+#pragma unroll
+        for (int b2 = 0; b2 < 2; ++b2)
+#pragma unroll
+            for (int cc = 0; cc < NCH; ++cc) ptx::tmem_fill_32x32(lane_taddr + b2 * TILE_M + cc * 32, ACC_BIAS_BITS);
+        ptx::tmem_st_wait();
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) {
+            ptx::mbar_arrive(bar(ACC_EMPTY + 0));
+            ptx::mbar_arrive(bar(ACC_EMPTY + 1));
+        }
         uint32_t it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
@@ -234,30 +262,56 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 if (g + 1 < G) sw_bits = __ldg(reinterpret_cast<const uint16_t*>(sw_ptr + (size_t)(g + 1) * BLOB_BYTES));
                 if (!(ok = ptx::mbar_wait(bar(ACC_FULL + buf), pa, abort_flag))) break;
                 ptx::tc_fence_after_sync();
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * TILE_M + h * C::HALF;
+                const uint32_t taddr = lane_taddr + buf * TILE_M;
+                uint32_t v[2][32];
+                ptx::tmem_ld_32x32(taddr, v[0]);
+                ptx::tmem_ld_wait();
 #pragma unroll
-                for (int ch = 0; ch < C::HALF / 32; ++ch) {
-                    uint32_t v[32];
-                    ptx::tmem_ld_32x32(taddr + ch * 32, v);
-                    ptx::tmem_ld_wait();
+                for (int ch = 0; ch < NCH; ++ch) {
+                    if (ch + 1 < NCH) {
+                        ptx::tmem_ld_32x32(taddr + (ch + 1) * 32, v[(ch + 1) & 1]);     // in flight during the math below
+                    } else {
+                        // every column of this buffer is in registers: start re-arming it (completion is
+                        // awaited after the math of the last chunk)
+#pragma unroll
+                        for (int cc = 0; cc < NCH; ++cc) ptx::tmem_fill_32x32(taddr + cc * 32, ACC_BIAS_BITS);
+                    }
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        facc[ch * 32 + i] = fmaf(sw, (float)(int)v[i], facc[ch * 32 + i]);
+                        const float d = __uint_as_float(v[ch & 1][i]) - 12582912.0f;       // exact: D as a float
+                        facc[ch * 32 + i] = fmaf(sw, d, facc[ch * 32 + i]);
                         if (DEBUG) {
                             const int m = m_base + ch * 32 + i;
-                            if (m < M) debug_partials[((size_t)m * G + g) * N + n] = (int)v[i];
+                            if (m < M) debug_partials[((size_t)m * G + g) * N + n] = (int)(v[ch & 1][i] - ACC_BIAS_BITS);
                         }
                     }
+                    if (ch + 1 < NCH) ptx::tmem_ld_wait();
                 }
+                ptx::tmem_st_wait();                       // the buffer is armed again: hand it back to the MMA warp
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(bar(ACC_EMPTY + buf));
             }
             if (!ok) break;
+            // Epilogue: token scale, bf16, and a transpose through shared memory so that global
+            // stores are 16 bytes per lane along the channel dimension (a thread owns a channel,
+            // the output is token-major).  Blocks of 32 tokens x this warp's 32 channels.
+            uint8_t* ob = smem + C::OUT_OFF + (warp - WARP_DRAIN0) * 2048;
+            __nv_bfloat16* yrow = y + (size_t)ntile * TILE_N + q * 32 + 8 * (lane & 3);
 #pragma unroll
-            for (int i = 0; i < C::HALF; ++i) {   // fully unrolled: facc must stay in registers
-                const int m = m_base + i;
-                if (m < M) y[(size_t)m * N + n] = __float2bfloat16_rn(facc[i] * sa_w[i]);
+            for (int b2 = 0; b2 < C::HALF / 32; ++b2) {
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    reinterpret_cast<__nv_bfloat16*>(ob + i * 64)[lane] = __float2bfloat16_rn(facc[b2 * 32 + i] * sa_w[b2 * 32 + i]);
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = (lane >> 2) + 8 * i;
+                    const int m = m_base + b2 * 32 + row;
+                    const uint4 val = *reinterpret_cast<const uint4*>(ob + row * 64 + 16 * (lane & 3));
+                    if (m < M) *reinterpret_cast<uint4*>(yrow + (size_t)m * N) = val;
+                }
             }
         }
     }

@@ -44,17 +44,34 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// same, but lets the hardware park the warp for up to `hint_ns` while the phase is pending, so
+// that a waiting role does not burn issue slots the working warps of the SM need
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
+    return ok != 0;
+}
 
-// Bounded wait: polls until the phase with the given parity completes, `*abort_flag`
-// (shared memory, set by any thread of the CTA that gave up) becomes non-zero, or about
-// `limit_ns` of wall time passes.  Returns false when it gave up; never spins forever.
+// Bounded wait: returns true once the phase with the given parity has completed; returns false
+// when `*abort_flag` (shared memory, set by any thread of the CTA that gave up) is non-zero or
+// about WAIT_LIMIT_NS of wall time have passed (it then sets the flag).  Never waits forever.
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // 2 s: orders of magnitude above any real wait
+constexpr uint32_t PARK_NS = 20000;                  // longest single park
+#ifndef W4A8_WAIT_BACKOFF_NS
+#define W4A8_WAIT_BACKOFF_NS 40
+#endif
+constexpr uint32_t WAIT_BACKOFF_NS = W4A8_WAIT_BACKOFF_NS;
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
     uint64_t t0 = 0;
     for (uint32_t spin = 1;; ++spin) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 0x3FF) == 0) {
+        if (mbar_try_wait_parked(bar, parity, PARK_NS)) return true;
+        __nanosleep(WAIT_BACKOFF_NS);            // leave the issue slots to the warps that have work
+        if ((spin & 0xF) == 0) {
             if (*abort_flag) return false;
             uint64_t now = globaltimer_ns();
             if (t0 == 0) t0 = now;
@@ -165,6 +182,33 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
+}
+// 32 lanes x 16 consecutive 32-bit columns
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+// fill 32 lanes x 16 consecutive columns with one 32-bit value
+__device__ __forceinline__ void tmem_fill_32x16(uint32_t taddr, uint32_t v) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
+        ::"r"(taddr), "r"(v) : "memory");
+}
+// fill 32 lanes x 32 consecutive columns with one 32-bit value
+__device__ __forceinline__ void tmem_fill_32x32(uint32_t taddr, uint32_t v) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, "
+        "%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
+        ::"r"(taddr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() {
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
