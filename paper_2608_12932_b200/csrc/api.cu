@@ -111,7 +111,7 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
                            int32_t* debug_partials, void* stream) {
     if (!shape_ok(N, K, group) || M < 0) return W4A8_ERR_SHAPE;
     if (path != W4A8_PATH_AUTO && path != W4A8_PATH_SPLITK && path != W4A8_PATH_TCGEN05 &&
-        path != W4A8_PATH_SPLITK_WORKSPACE)
+        path != W4A8_PATH_SPLITK_WORKSPACE && path != W4A8_PATH_TCGEN05_PAIR)
         return W4A8_ERR_SHAPE;
     if ((path == W4A8_PATH_SPLITK || path == W4A8_PATH_SPLITK_WORKSPACE) && M > SPLITK_MAX_M) return W4A8_ERR_SHAPE;
     if (M == 0) return W4A8_OK;
@@ -129,7 +129,8 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
     else if (path == W4A8_PATH_SPLITK || (path == W4A8_PATH_AUTO && M <= SPLITK_MAX_M))
         e = launch_gemm_cluster(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
     else
-        e = launch_gemm_tcgen05(qa, sa, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
+        e = launch_gemm_tcgen05(qa, sa, packed_w, y_bf16, M, N, K, workspace, debug_partials, st,
+                                path == W4A8_PATH_TCGEN05_PAIR);
     return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
 

@@ -55,6 +55,6 @@ cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int3
                                 cudaStream_t stream);
 cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
                                 int M, int N, int K, void* workspace, int32_t* debug_partials,
-                                cudaStream_t stream);
+                                cudaStream_t stream, bool want_pair);
 
 }  // namespace w4a8

@@ -18,7 +18,7 @@ from tests.gpu_util import DeviceLayer, bits, t_u16
 pytestmark = pytest.mark.gpu
 
 PATHS = {"splitk": B.PATH_SPLITK, "splitk_ws": B.PATH_SPLITK_WORKSPACE, "tcgen05": B.PATH_TCGEN05,
-         "auto": B.PATH_AUTO}
+         "tcgen05_pair": B.PATH_TCGEN05_PAIR, "auto": B.PATH_AUTO}
 
 
 def check_case(case, layer, M, path, debug=True, rows=None):
@@ -95,6 +95,19 @@ def test_splitk_token_counts(mid_case, M, path):
 def test_tcgen05_token_counts(mid_case, M):
     case, layer = mid_case
     check_case(case, layer, M, "tcgen05")
+
+
+@pytest.fixture(scope="module")
+def pair_case():
+    case = wl.make_layer(1024, 512, 36, 600)          # N a multiple of 256: M > 128 runs CTA pairs
+    return case, DeviceLayer(case, 600)
+
+
+@pytest.mark.parametrize("M", [129, 200, 256, 257, 384, 385, 520, 600])
+def test_tcgen05_cta_pair_token_counts(pair_case, M):
+    case, layer = pair_case
+    check_case(case, layer, M, "tcgen05_pair")
+    check_case(case, layer, M, "tcgen05", debug=False)
 
 
 @pytest.mark.parametrize("M", [1, 8, 64, 65, 300])
