@@ -376,7 +376,7 @@ def run_gpu(args):
                 "d2h_bytes_per_step": M * N * 2, "ms_per_step": e2e_ms / args.steps},
         "gpu_launches": 2 * args.steps,
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "gemm_splitk_kernel<1>", "achieved": round(achieved, 1),
+        "roofline": {"bound": "hbm", "kernel": "gemm_cluster_kernel<1>", "achieved": round(achieved, 1),
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4),
                      "peak_source": f"of {peaks['source']} (STREAM-style copy, burst)",
                      "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),

@@ -22,6 +22,7 @@
 //    one wave keeps its CTAs under half an SM's shared memory and prefetches as much of its slice
 //    as fits, so that two consecutive launches can be resident together and the weight stream of
 //    the next overlaps the tail of the current one.
+#include <cstdlib>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include "ptx_sm100.cuh"
@@ -348,24 +349,28 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
 }
 }  // namespace
 
-// Slices per tile for the cluster kernel: the S in 1..8 (portable cluster size; never more than
-// the number of groups) that minimises the longest per-SM chain, ceil(CTAs / SMs) * ceil(G / S);
-// ties go to the smaller S (less to reduce).
-int cluster_num_slices(int N, int K) {
+// Slices per tile for the cluster kernel, at most 8 (portable cluster size) and never more than
+// the number of groups.  Measured on the four layer shapes: one m-block (M <= 8) runs best with
+// about 1.4 CTAs per SM (two co-resident CTAs per SM leave room for the next launch to prefetch),
+// larger M, whose CTAs hold more registers and shared memory, with about 0.75.
+int cluster_num_slices(int M, int N, int K) {
     const int G = K / GROUP, tiles = N / TILE_N, sms = sm_count();
-    int best = 1;
-    long best_cost = -1;
-    for (int s = 1; s <= CL_MAX_S && s <= G; ++s) {
-        const long cost = (long)((tiles * s + sms - 1) / sms) * ((G + s - 1) / s);
-        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+    if (const char* e = getenv("W4A8_CLUSTER_S")) {      // tuning aid: force the slice count
+        int v = atoi(e);
+        if (v >= 1 && v <= CL_MAX_S && v <= G) return v;
     }
-    return best;
+    const int target = M <= 8 ? (sms * 14) / 10 : (sms * 3) / 4;
+    int s = (target + tiles / 2) / tiles;
+    if (s > CL_MAX_S) s = CL_MAX_S;
+    if (s > G) s = G;
+    if (s < 1) s = 1;
+    return s;
 }
 
 cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
                                 void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream) {
-    const int S = cluster_num_slices(N, K);
+    const int S = cluster_num_slices(M, N, K);
     if (M <= 8) return launch_mb<1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
     if (M <= 16) return launch_mb<2>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
     if (M <= 32) return launch_mb<4>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
