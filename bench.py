@@ -180,6 +180,21 @@ class Timer:
         return g, times
 
 
+def max_over_ranks(ms, dist, device):
+    """A time measured on every rank -> the slowest rank's (what a replicated job waits for)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(ms)
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(bytes_per_step, steps, world, ms):
+    """Replicas only: every rank runs the same steps on its own GPU; the job's throughput is the sum."""
+    return bytes_per_step * steps * world / (ms * 1e-3) / 1e9
+
+
 def copies_for(nbytes, l2_bytes):
     return int(np.ceil(2.0 * l2_bytes / nbytes)) + 1
 
@@ -308,12 +323,9 @@ def run_gpu(args):
         torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else None
     B.w4a8_check_status(ws)
-    if world > 1:
-        t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dist if world > 1 else None, "cuda")
     sbytes = step_bytes(M, N, K)
-    value = sbytes * args.steps * world / (ms_total * 1e-3) / 1e9
+    value = whole_job_gbs(sbytes, args.steps, world, ms_total)
 
     # ---- roofline of the dominant kernel: the split-K GEMM alone, same rotation, K launches
     def gemm_only():
@@ -342,11 +354,8 @@ def run_gpu(args):
     g_e2e, et = timer.graph_ms(e2e_steps, replays=3, warm=2)
     barrier()
     e2e_ms = float(np.median(et))
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = sbytes * args.steps * world / (e2e_ms * 1e-3) / 1e9
+    e2e_ms = max_over_ranks(e2e_ms, dist if world > 1 else None, "cuda")
+    e2e_value = whole_job_gbs(sbytes, args.steps, world, e2e_ms)
     e2e_ok, _ = onp.within_tolerance(y_host.view(torch.int16).numpy().view(np.uint16), ref["ref"])
     parity["e2e_within_tolerance"] = e2e_ok
 
