@@ -441,8 +441,8 @@ def run_shape(args):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one split-K GEMM launch at the headline shape,
-# from the ncu capture summarised under profiles/ (None until a capture exists)
-TRAFFIC_BYTES_PER_LAUNCH = None
+# from the ncu capture summarised in profiles/gemm_cluster_qkv_M8.md
+TRAFFIC_BYTES_PER_LAUNCH = 13132288
 
 
 def main():
