@@ -25,6 +25,38 @@ w4a8_status arch_check() {
     return cached[dev] == 1 ? W4A8_OK : W4A8_ERR_ARCH;
 }
 
+}  // namespace
+
+namespace w4a8 {
+
+int device_sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (!cached[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+// Between 33 and 64 tokens both kernel families are valid.  Measured on B200 (microseconds, cold
+// weights): the streaming kernel costs about 7 + 2.0 x (blobs per SM), because above 32 tokens it
+// walks the token blocks twice; the tensor-core kernel costs about 2 + 0.7 x groups x (tiles per
+// CTA), its unpack warps being the limit whatever the token count.  Pick the smaller estimate.
+bool small_m_prefers_tcgen05(int M, int N, int K, int sms) {
+    if (M <= 32 || M > SPLITK_MAX_M) return M > SPLITK_MAX_M;
+    const long G = K / GROUP, tiles = N / TILE_N;
+    const long streaming_ns = 7000 + 2030 * (tiles * G) / sms;
+    const long tensor_ns = 2000 + 700 * G * ((tiles + sms - 1) / sms);
+    return tensor_ns < streaming_ns;
+}
+
+}  // namespace w4a8
+
+namespace {
+
 size_t slices_bytes(int M, int N, int K) {
     const int m = M < SPLITK_MAX_M ? M : SPLITK_MAX_M;
     const int S = splitk_num_slices(m, N, K);
@@ -126,7 +158,7 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
     cudaError_t e;
     if (path == W4A8_PATH_SPLITK_WORKSPACE)
         e = launch_gemm_splitk(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
-    else if (path == W4A8_PATH_SPLITK || (path == W4A8_PATH_AUTO && M <= SPLITK_MAX_M))
+    else if (path == W4A8_PATH_SPLITK || (path == W4A8_PATH_AUTO && !small_m_prefers_tcgen05(M, N, K, device_sm_count())))
         e = launch_gemm_cluster(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
     else
         e = launch_gemm_tcgen05(qa, sa, packed_w, y_bf16, M, N, K, workspace, debug_partials, st,

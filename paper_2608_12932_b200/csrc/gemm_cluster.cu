@@ -274,18 +274,6 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
     }
 }
 
-int sm_count() {
-    static int cached[64] = {0};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-    if (!cached[dev]) {
-        int n = 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-        cached[dev] = n;
-    }
-    return cached[dev];
-}
-
 template <int MB>
 cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed, void* y,
                       int M, int N, int K, int S, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
@@ -293,7 +281,7 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
     const int ng_max = (G + S - 1) / S;
     // shared-memory budget per CTA: a launch of at most one wave leaves room for the next launch's
     // CTAs on the same SMs; larger launches share the SM between ceil(CTAs/SMs) CTAs of their own
-    const int ctas = (N / TILE_N) * S, sms = sm_count();
+    const int ctas = (N / TILE_N) * S, sms = device_sm_count();
     const int waves = (ctas + sms - 1) / sms;
     int budget = waves <= 1 ? 110 * 1024 : (220 * 1024) / waves;
     if (budget < 40 * 1024) budget = 40 * 1024;
@@ -354,7 +342,7 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
 // about 1.4 CTAs per SM (two co-resident CTAs per SM leave room for the next launch to prefetch),
 // larger M, whose CTAs hold more registers and shared memory, with about 0.75.
 int cluster_num_slices(int M, int N, int K) {
-    const int G = K / GROUP, tiles = N / TILE_N, sms = sm_count();
+    const int G = K / GROUP, tiles = N / TILE_N, sms = device_sm_count();
     if (const char* e = getenv("W4A8_CLUSTER_S")) {      // tuning aid: force the slice count
         int v = atoi(e);
         if (v >= 1 && v <= CL_MAX_S && v <= G) return v;

@@ -425,18 +425,12 @@ cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed
     cudaError_t te = make_qa_tensor_map(&tmap, qa, M, K, C::B_ROWS);
     if (te != cudaSuccess) return te;
 
-    int dev = 0, sms = 0;
+    int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    static int sm_count[64] = {0};
     static bool attr_done[64] = {false};
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (!sm_count[dev]) {
-        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-        sm_count[dev] = sms;
-    }
-    sms = sm_count[dev];
+    const int sms = device_sm_count();
     if (!attr_done[dev]) {
         e = cudaFuncSetAttribute(gemm_tcgen05_kernel<TILE_M, DEBUG, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  C::SMEM_ALLOC);
@@ -468,20 +462,46 @@ cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed
 
 }  // namespace
 
+// Token-tile height for an [M, N] problem.  A CTA's time per tile is dominated by unpacking the
+// tile's weights, which does not depend on the tile height: measured on B200 a 64-, 128- and
+// 256-token tile cost 1 : 1.13 : 1.47.  The persistent grid runs ceil(tiles / SMs) tiles per CTA,
+// so the height with the smallest (tiles per CTA) x (cost per tile) wins: tall tiles when there
+// are several waves of them, short ones when a tall tiling would leave SMs idle.
+int tcgen05_tile_m(int M, int N, int sms) {
+    const int heights[3] = {256, 128, 64};
+    const int cost[3] = {147, 113, 100};
+    const int n_tiles = N / TILE_N;
+    int best = 64;
+    long best_cost = -1;
+    for (int i = 0; i < 3; ++i) {
+        if (heights[i] > 64 && M <= heights[i] / 2) continue;       // half the height already covers M in one tile
+        const long tiles = (long)((M + heights[i] - 1) / heights[i]) * n_tiles;
+        const long c = ((tiles + sms - 1) / sms) * cost[i];
+        if (best_cost < 0 || c < best_cost) { best_cost = c; best = heights[i]; }   // ties go to the taller tile
+    }
+    return best;
+}
+
+namespace {
+template <bool DEBUG>
+cudaError_t launch_height(int tile_m, bool pair, const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
+                          int M, int N, int K, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
+    if (pair) return launch_tile<256, DEBUG, true>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+    if (tile_m == 64) return launch_tile<64, DEBUG, false>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+    if (tile_m == 128) return launch_tile<128, DEBUG, false>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+    return launch_tile<256, DEBUG, false>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+}
+}  // namespace
+
 cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
                                 int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream, bool want_pair) {
     const bool pair = want_pair && M > 128 && N % (2 * TILE_N) == 0;
-    if (debug_partials) {
-        if (M <= 64) return launch_tile<64, true, false>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
-        if (M <= 128) return launch_tile<128, true, false>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
-        if (pair) return launch_tile<256, true, true>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
-        return launch_tile<256, true, false>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
-    }
-    if (M <= 64) return launch_tile<64, false, false>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
-    if (M <= 128) return launch_tile<128, false, false>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
-    if (pair) return launch_tile<256, false, true>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
-    return launch_tile<256, false, false>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+    const int sms = device_sm_count();
+    const int tile_m = tcgen05_tile_m(M, N, sms);
+    if (debug_partials)
+        return launch_height<true>(tile_m, pair, qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+    return launch_height<false>(tile_m, pair, qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
 }
 
 }  // namespace w4a8

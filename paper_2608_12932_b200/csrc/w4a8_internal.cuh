@@ -49,6 +49,7 @@ cudaError_t launch_unpack_weights(const void* packed, int N, int K, uint8_t* qw,
 cudaError_t launch_gemm_splitk(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
                                void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
                                cudaStream_t stream);
+int device_sm_count();                       // SMs of the current device (cached per device)
 int cluster_num_slices(int M, int N, int K);
 cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
                                 void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
@@ -56,5 +57,7 @@ cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int3
 cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
                                 int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream, bool want_pair);
+int tcgen05_tile_m(int M, int N, int sms);    // token-tile height the tcgen05 launcher picks
+bool small_m_prefers_tcgen05(int M, int N, int K, int sms);
 
 }  // namespace w4a8
