@@ -161,8 +161,7 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
     else if (path == W4A8_PATH_SPLITK || (path == W4A8_PATH_AUTO && !small_m_prefers_tcgen05(M, N, K, device_sm_count())))
         e = launch_gemm_cluster(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
     else
-        e = launch_gemm_tcgen05(qa, sa, packed_w, y_bf16, M, N, K, workspace, debug_partials, st,
-                                path == W4A8_PATH_TCGEN05_PAIR);
+        e = launch_gemm_tcgen05(qa, sa, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
     return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
 
