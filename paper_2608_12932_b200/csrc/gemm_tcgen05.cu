@@ -50,6 +50,7 @@ namespace {
 
 constexpr int TC_THREADS = 512;
 constexpr int WARP_PRODUCER = 0, WARP_MMA = 1, WARP_RAW_PRODUCER = 2, WARP_MMA_ODD = 3, WARP_UNPACK0 = 4, WARP_DRAIN0 = 8;
+constexpr int PRODUCER_LANES = 4;                // threads per copy producer
 constexpr int DONE_RING = 8;                     // "group finished" barriers; every role stays within 8 groups of the others
 constexpr int NUM_UNPACK_WARPS = 4, NUM_DRAIN_WARPS = 8;
 constexpr int RAW_STRIDE = 8576;                 // BLOB_BYTES rounded up to a multiple of 128
@@ -64,7 +65,8 @@ template <int TILE_M>
 struct Cfg {
     static constexpr int B_BYTES = TILE_M * GROUP;                            // one activation stage
     static constexpr int SB = TILE_M > 128 ? 5 : (TILE_M == 128 ? 6 : 8);     // activation stages
-    static constexpr int SR = 6;                                              // packed-blob stages
+    static constexpr int SR = TILE_M > 128 ? 8 : (TILE_M == 128 ? 12 : 16);   // packed-blob stages: a short tile finishes a group
+                                                                              // quickly, so more blobs must be in flight to cover HBM latency
     static constexpr int SA_MAX = (TMEM_COLS - 2 * TILE_M) / A_COLS;
     static constexpr int SA = SA_MAX > 4 ? 4 : SA_MAX;                        // weight stages in TMEM
     static constexpr int A_COL0 = 2 * TILE_M;                                 // first weight column (after two accumulators)
@@ -151,7 +153,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
 
     if (warp < 4) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
-        if (warp == WARP_PRODUCER && lane == 0) {
+        // A producer iteration is a chain of dependent round trips (barrier probe, expect-tx, copy
+        // issue) of several hundred cycles; PRODUCER_LANES lanes take the pipeline steps round-robin so
+        // that the chains overlap.
+        if (warp == WARP_PRODUCER && lane < PRODUCER_LANES) {
             // ------------------------------------------------ producer: activation tiles ----
             uint32_t it = 0;
             bool ok = true;
@@ -159,6 +164,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 int ntile, mtile;
                 tile_of(tile, ntile, mtile);
                 for (int g = 0; g < G; ++g, ++it) {
+                    if ((int)(it % PRODUCER_LANES) != lane) continue;
                     const uint32_t sb = it % C::SB;
                     if (it >= (uint32_t)C::SB && !(ok = ptx::mbar_wait(done_bar(it - C::SB), done_parity(it - C::SB), abort_flag))) break;
                     ptx::mbar_arrive_expect_tx(bar(B_FULL + sb), C::B_BYTES);
@@ -170,7 +176,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 const uint64_t t0 = ptx::globaltimer_ns();
                 while (ptx::globaltimer_ns() - t0 < 200000ull) {}
             }
-        } else if (warp == WARP_RAW_PRODUCER && lane == 0) {
+        } else if (warp == WARP_RAW_PRODUCER && lane < PRODUCER_LANES) {
             // --------------------------------------------------- producer: packed blobs ----
             uint32_t it = 0;
             bool ok = true;
@@ -179,6 +185,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 tile_of(tile, ntile, mtile);
                 const uint8_t* src = packed + (size_t)ntile * G * BLOB_BYTES;
                 for (int g = 0; g < G; ++g, ++it) {
+                    if ((int)(it % PRODUCER_LANES) != lane) continue;
                     const uint32_t sr = it % C::SR, pr = (it / C::SR) & 1;
                     if (!(ok = ptx::mbar_wait(bar(RAW_EMPTY + sr), pr ^ 1, abort_flag))) break;
                     ptx::mbar_arrive_expect_tx(bar(RAW_FULL + sr), BLOB_BYTES);
@@ -304,28 +311,25 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 if (!(ok = ptx::mbar_wait_hot(done_bar(it), done_parity(it), abort_flag))) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t taddr = lane_taddr + buf * TILE_M;
-                uint32_t v[2][32];
-                auto load_chunk = [&](int ch) {
-                    if (ch == C::NCH - 1 && C::LAST == 8) ptx::tmem_ld_32x8(taddr + ch * 32, reinterpret_cast<uint32_t(&)[8]>(v[ch & 1]));
-                    else ptx::tmem_ld_32x32(taddr + ch * 32, v[ch & 1]);
-                };
-                load_chunk(0);
-                ptx::tmem_ld_wait();
+                // All of this warp's columns go to registers with back-to-back loads, then the buffer is
+                // handed back: the MMA -> drain -> MMA round trip of a buffer, not the arithmetic
+                // below, sets the pace of the pipeline.
+                uint32_t v[C::NCH][32];
 #pragma unroll
                 for (int ch = 0; ch < C::NCH; ++ch) {
-                    if (ch + 1 < C::NCH) {
-                        load_chunk(ch + 1);                               // in flight during the arithmetic below
-                    } else {
-                        // every column of this buffer is in registers: hand it back to the MMA warp
-                        // before the arithmetic on the last chunk
-                        ptx::tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(bar(ACC_EMPTY + buf));
-                    }
+                    if (ch == C::NCH - 1 && C::LAST == 8) ptx::tmem_ld_32x8(taddr + ch * 32, reinterpret_cast<uint32_t(&)[8]>(v[ch]));
+                    else ptx::tmem_ld_32x32(taddr + ch * 32, v[ch]);
+                }
+                ptx::tmem_ld_wait();
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar(ACC_EMPTY + buf));
+#pragma unroll
+                for (int ch = 0; ch < C::NCH; ++ch) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         if (ch * 32 + i < C::W) {
-                            const int32_t di = (int32_t)v[ch & 1][i];
+                            const int32_t di = (int32_t)v[ch][i];
                             facc[ch * 32 + i] = fmaf(sw, (float)di, facc[ch * 32 + i]);     // exact convert: |D| < 2^24
                             if (DEBUG) {
                                 const int m = m_base + ch * 32 + i;
@@ -333,7 +337,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                             }
                         }
                     }
-                    if (ch + 1 < C::NCH) ptx::tmem_ld_wait();
                 }
             }
             if (!ok) break;
