@@ -55,10 +55,8 @@ typedef enum {
     W4A8_PATH_SPLITK = 1,    /* weight-streaming split-K kernel, slices reduced inside a
                                 thread-block cluster through distributed shared memory (M <= 64) */
     W4A8_PATH_TCGEN05 = 2,   /* TMA + tcgen05.mma kind::i8 + TMEM kernel (any M)             */
-    W4A8_PATH_SPLITK_WORKSPACE = 3, /* split-K kernel that reduces its slices through the global
+    W4A8_PATH_SPLITK_WORKSPACE = 3  /* split-K kernel that reduces its slices through the global
                                 workspace (M <= 64); what w4a8_gemm_static_scratch runs        */
-    W4A8_PATH_TCGEN05_PAIR = 4  /* tcgen05 kernel with CTA pairs (cta_group::2) where the shape
-                                allows (M > 128, N % 256 == 0), else as W4A8_PATH_TCGEN05       */
 } w4a8_path;
 
 const char* w4a8_status_string(w4a8_status s);

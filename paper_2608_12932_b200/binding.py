@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libw4a8.so")
 
 GROUP = 128
 OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(8)
-PATH_AUTO, PATH_SPLITK, PATH_TCGEN05, PATH_SPLITK_WORKSPACE, PATH_TCGEN05_PAIR = 0, 1, 2, 3, 4
+PATH_AUTO, PATH_SPLITK, PATH_TCGEN05, PATH_SPLITK_WORKSPACE = 0, 1, 2, 3
 WORKSPACE_HEADER_BYTES = 4096
 
 EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w4a8_workspace_init",

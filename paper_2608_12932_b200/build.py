@@ -39,9 +39,9 @@ def check_ptxas(report):
                          r".*?Used (\d+) registers", report, re.S):
         name, spill, regs = m.group(1), int(m.group(2)), int(m.group(3))
         limit = 64                                # a few stray registers are tolerable, an accumulator array is not
-        m2 = re.search(r"gemm_tcgen05_kernelILi\d+ELb(\d)ELb(\d)E", name)
-        if m2 and (m2.group(1) == "1" or m2.group(2) == "1"):
-            limit = 1024                          # debug (partials dump) and CTA-pair instantiations may spill
+        m2 = re.search(r"gemm_tcgen05_kernelILi\d+ELb(\d)E", name)
+        if m2 and m2.group(1) == "1":
+            limit = 1024                          # the debug instantiations (partials dump) may spill
         if spill > limit and "gemm_" in name:
             problems.append(f"{name}: {spill} bytes of spill stores")
         if "gemm_tcgen05_kernel" in name and regs != 128:

@@ -41,15 +41,16 @@ int device_sm_count() {
     return cached[dev];
 }
 
-// Between 33 and 64 tokens both kernel families are valid.  Measured on B200 (microseconds, cold
-// weights): the streaming kernel costs about 7 + 2.0 x (blobs per SM), because above 32 tokens it
-// walks the token blocks twice; the tensor-core kernel costs about 2 + 0.7 x groups x (tiles per
-// CTA), its unpack warps being the limit whatever the token count.  Pick the smaller estimate.
+// Between 17 and 64 tokens both kernel families are valid.  Measured on B200 (nanoseconds, cold
+// weights): the streaming kernel costs about 3000 + 950 x (blobs per SM) up to 32 tokens and, because
+// it then walks the token blocks twice, 7000 + 2030 x (blobs per SM) above; the tensor-core kernel
+// costs about 4000 + 440 x groups x (tiles per CTA) whatever the token count.  Pick the smaller estimate.
 bool small_m_prefers_tcgen05(int M, int N, int K, int sms) {
-    if (M <= 32 || M > SPLITK_MAX_M) return M > SPLITK_MAX_M;
+    if (M <= 16 || M > SPLITK_MAX_M) return M > SPLITK_MAX_M;
     const long G = K / GROUP, tiles = N / TILE_N;
-    const long streaming_ns = 7000 + 2030 * (tiles * G) / sms;
-    const long tensor_ns = 2000 + 700 * G * ((tiles + sms - 1) / sms);
+    const long blobs_per_sm = (tiles * G) / sms;
+    const long streaming_ns = M <= 32 ? 3000 + 950 * blobs_per_sm : 7000 + 2030 * blobs_per_sm;
+    const long tensor_ns = 4000 + 440 * G * ((tiles + sms - 1) / sms);
     return tensor_ns < streaming_ns;
 }
 
@@ -143,7 +144,7 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
                            int32_t* debug_partials, void* stream) {
     if (!shape_ok(N, K, group) || M < 0) return W4A8_ERR_SHAPE;
     if (path != W4A8_PATH_AUTO && path != W4A8_PATH_SPLITK && path != W4A8_PATH_TCGEN05 &&
-        path != W4A8_PATH_SPLITK_WORKSPACE && path != W4A8_PATH_TCGEN05_PAIR)
+        path != W4A8_PATH_SPLITK_WORKSPACE)
         return W4A8_ERR_SHAPE;
     if ((path == W4A8_PATH_SPLITK || path == W4A8_PATH_SPLITK_WORKSPACE) && M > SPLITK_MAX_M) return W4A8_ERR_SHAPE;
     if (M == 0) return W4A8_OK;

@@ -57,7 +57,7 @@ constexpr int RAW_STRIDE = 8576;                 // BLOB_BYTES rounded up to a m
 constexpr int A_COLS = GROUP / 4;                // 32 TMEM columns hold one group of a weight row (4 bytes per column)
 constexpr int TMEM_COLS = 512;
 // relative cost of one 208-, 128-, 64-token tile (same channels, same K), measured
-constexpr int TC_COST_208 = 140, TC_COST_128 = 113, TC_COST_64 = 100;
+constexpr int TC_COST_208 = 148, TC_COST_128 = 123, TC_COST_64 = 100;
 
 // Shared-memory rings.  The activation tile comes from L2 through TMA with a latency of roughly
 // 2000 cycles, the packed blob from HBM likewise: both rings are deep enough to cover it.

@@ -17,8 +17,7 @@ from tests.gpu_util import DeviceLayer, bits, t_u16
 
 pytestmark = pytest.mark.gpu
 
-PATHS = {"splitk": B.PATH_SPLITK, "splitk_ws": B.PATH_SPLITK_WORKSPACE, "tcgen05": B.PATH_TCGEN05,
-         "tcgen05_pair": B.PATH_TCGEN05_PAIR, "auto": B.PATH_AUTO}
+PATHS = {"splitk": B.PATH_SPLITK, "splitk_ws": B.PATH_SPLITK_WORKSPACE, "tcgen05": B.PATH_TCGEN05, "auto": B.PATH_AUTO}
 
 
 def check_case(case, layer, M, path, debug=True, rows=None):
@@ -91,23 +90,27 @@ def test_splitk_token_counts(mid_case, M, path):
     check_case(case, layer, M, path)
 
 
-@pytest.mark.parametrize("M", [1, 16, 64, 65, 128, 129, 255, 256, 257, 300, 520, 600])
+# token tiles are 64, 128 or 208 rows; a 208-row tile is drained in column pieces of 32, 32, 32 and 8
+@pytest.mark.parametrize("M", [1, 16, 64, 65, 96, 97, 104, 105, 128, 129, 200, 207, 208, 209, 255, 256, 257, 300, 415, 416, 417,
+                               520, 600])
 def test_tcgen05_token_counts(mid_case, M):
     case, layer = mid_case
     check_case(case, layer, M, "tcgen05")
 
 
 @pytest.fixture(scope="module")
-def pair_case():
-    case = wl.make_layer(1024, 512, 36, 600)          # N a multiple of 256: M > 128 runs CTA pairs
-    return case, DeviceLayer(case, 600)
+def wide_case():
+    case = wl.make_layer(1024, 5120, 36, 1000)        # 40 channel tiles
+    return case, DeviceLayer(case, 1000)
 
 
-@pytest.mark.parametrize("M", [129, 200, 256, 257, 384, 385, 520, 600])
-def test_tcgen05_cta_pair_token_counts(pair_case, M):
-    case, layer = pair_case
-    check_case(case, layer, M, "tcgen05_pair")
-    check_case(case, layer, M, "tcgen05", debug=False)
+@pytest.mark.parametrize("M", [300, 417, 624, 625, 1000])
+def test_tcgen05_tile_heights_and_waves(wide_case, M):
+    """Token counts on both sides of the dispatch's choice between 128- and 208-row tiles, with more
+    tiles than SMs for the larger ones (a CTA then walks several tiles)."""
+    case, layer = wide_case
+    check_case(case, layer, M, "tcgen05")
+    check_case(case, layer, M, "auto", debug=False)
 
 
 @pytest.mark.parametrize("M", [1, 8, 64, 65, 300])
