@@ -129,9 +129,25 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
                            int32_t* debug_partials, void* stream);
 
 /*
+ * The whole path on device buffers: y = W4A8 linear of bf16 activations, i.e. w4a8_quantize_act
+ * followed by w4a8_gemm on the same stream (Sec. 3.4); two kernel launches, chained with
+ * programmatic dependent launch so that the GEMM's weight stream starts under the quantiser.
+ * (A single-kernel form, in which the small-M GEMM quantises its own activations, was built and
+ * measured slower: every CTA then repeats the row-maximum and division work of the quantiser.)
+ *   x_bf16   [M,K] bf16 bits, contiguous, 16-byte aligned
+ *   y_bf16   [M,N] bf16 bits, fully overwritten
+ *   qa, sa, asum   as for w4a8_quantize_act: required scratch, holding the quantised activations afterwards
+ * Same shape rules, workspace and status codes as w4a8_gemm.
+ */
+w4a8_status w4a8_linear(const void* x_bf16, const void* packed_w, void* y_bf16,
+                        int M, int N, int K, int group,
+                        int8_t* qa, uint16_t* sa, int32_t* asum,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The whole path for callers whose activations and results live in HOST memory (Sec. 3.5: a
  * pipeline stage is one graph launch fed from the host): enqueues, on `stream`, the copy of
- * x to the device, w4a8_quantize_act, w4a8_gemm, and the copy of y back to the host.
+ * x to the device, w4a8_linear, and the copy of y back to the host.
  *   x_host_bf16  HOST [M,K] bf16 (pinned memory makes the copies asynchronous)
  *   y_host_bf16  HOST [M,N] bf16, valid once `stream` has been synchronised by the caller
  *   x_dev, qa, sa, asum, y_dev   DEVICE staging buffers owned by the caller, sized and aligned

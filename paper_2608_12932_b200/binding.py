@@ -19,7 +19,7 @@ WORKSPACE_HEADER_BYTES = 4096
 
 EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w4a8_workspace_init",
            "w4a8_pack_weights", "w4a8_unpack_weights", "w4a8_quantize_act", "w4a8_gemm", "w4a8_gemm_path",
-           "w4a8_linear_host", "w4a8_gemm_static_scratch", "w4a8_check_status")
+           "w4a8_linear", "w4a8_linear_host", "w4a8_gemm_static_scratch", "w4a8_check_status")
 
 _lib = None
 
@@ -57,6 +57,8 @@ def lib():
         L.w4a8_gemm.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp, vp]
         L.w4a8_gemm_path.restype = ci
         L.w4a8_gemm_path.argtypes = [ci, vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp, vp]
+        L.w4a8_linear.restype = ci
+        L.w4a8_linear.argtypes = [vp, vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, sz, vp]
         L.w4a8_linear_host.restype = ci
         L.w4a8_linear_host.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.w4a8_gemm_static_scratch.restype = ci
@@ -172,6 +174,27 @@ def w4a8_gemm(qa, sa, asum, packed_w, N, workspace, group=GROUP, out=None, debug
     return out
 
 
+def w4a8_linear(x, packed_w, N, workspace, group=GROUP, out=None, scratch=None, stream=None):
+    """y bf16 [M,N] = W4A8 linear of bf16 activations [M,K]: quantise, then multiply (two kernels on
+    one stream).  `scratch` = (qa, sa, asum) buffers as w4a8_quantize_act returns them (allocated
+    here when absent); they hold the quantised activations afterwards."""
+    _dev(x, torch.bfloat16, "x"), _dev(packed_w, torch.uint8, "packed_w"), _dev(workspace, torch.uint8, "workspace")
+    M, K = x.shape
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+    else:
+        _dev(out, torch.bfloat16, "out")
+    if scratch is None:
+        scratch = (torch.empty((M, K), dtype=torch.int8, device=x.device),
+                   torch.empty((M,), dtype=torch.float16, device=x.device),
+                   torch.empty((M, max(K // group, 1)), dtype=torch.int32, device=x.device))
+    qa, sa, asum = scratch
+    _dev(qa, torch.int8, "qa"), _dev(sa, torch.float16, "sa"), _dev(asum, torch.int32, "asum")
+    _check(lib().w4a8_linear(_ptr(x), _ptr(packed_w), _ptr(out), M, N, K, group, _ptr(qa), _ptr(sa), _ptr(asum),
+                             _ptr(workspace), workspace.numel(), _stream(stream)), "w4a8_linear")
+    return out
+
+
 STATIC_SCRATCH_BYTES = 4096 + 4 * 1024 * 1024
 
 
@@ -218,9 +241,3 @@ class HostLinear:
                                       _ptr(self.asum), _ptr(self.y_dev), _ptr(self.workspace),
                                       self.workspace.numel(), _stream(stream)), "w4a8_linear_host")
         return y_host
-
-
-def w4a8_linear(x, packed_w, N, workspace, group=GROUP, stream=None):
-    """Convenience: quantise activations, then the GEMM (two library calls on one stream)."""
-    qa, sa, asum = w4a8_quantize_act(x, group, stream=stream)
-    return w4a8_gemm(qa, sa, asum, packed_w, N, workspace, group, stream=stream)

@@ -175,6 +175,17 @@ w4a8_status w4a8_gemm(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
                           workspace, workspace_bytes, debug_partials, stream);
 }
 
+w4a8_status w4a8_linear(const void* x_bf16, const void* packed_w, void* y_bf16,
+                        int M, int N, int K, int group,
+                        int8_t* qa, uint16_t* sa, int32_t* asum,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    if (!shape_ok(N, K, group) || M < 0) return W4A8_ERR_SHAPE;
+    if (M == 0) return W4A8_OK;
+    w4a8_status s = w4a8_quantize_act(x_bf16, M, K, group, qa, sa, asum, stream);
+    if (s != W4A8_OK) return s;
+    return w4a8_gemm(qa, sa, asum, packed_w, y_bf16, M, N, K, group, workspace, workspace_bytes, nullptr, stream);
+}
+
 w4a8_status w4a8_linear_host(const void* x_host_bf16, void* y_host_bf16,
                              int M, int N, int K, int group, const void* packed_w,
                              void* x_dev, int8_t* qa, uint16_t* sa, int32_t* asum, void* y_dev,
@@ -185,9 +196,7 @@ w4a8_status w4a8_linear_host(const void* x_host_bf16, void* y_host_bf16,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(x_dev, x_host_bf16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return W4A8_ERR_CUDA;
-    w4a8_status s = w4a8_quantize_act(x_dev, M, K, group, qa, sa, asum, stream);
-    if (s != W4A8_OK) return s;
-    s = w4a8_gemm(qa, sa, asum, packed_w, y_dev, M, N, K, group, workspace, workspace_bytes, nullptr, stream);
+    w4a8_status s = w4a8_linear(x_dev, packed_w, y_dev, M, N, K, group, qa, sa, asum, workspace, workspace_bytes, stream);
     if (s != W4A8_OK) return s;
     if (cudaMemcpyAsync(y_host_bf16, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return W4A8_ERR_CUDA;

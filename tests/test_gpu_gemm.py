@@ -275,3 +275,85 @@ def test_decoder_layer_sweep_sampled():
             assert ok, f"{lname} M={M}: worst |err|/bound = {ratio:.3f}"
         del layer
         torch.cuda.empty_cache()
+
+
+# ------------------------------------------- w4a8_linear: quantise + multiply, one call ---
+def _linear(case, layer, M):
+    x = t_u16(case["x"][:M], torch.bfloat16)
+    y = B.w4a8_linear(x, layer.packed, case["N"], layer.ws)
+    torch.cuda.synchronize()
+    B.w4a8_check_status(layer.ws)
+    return bits(y)
+
+
+@pytest.mark.parametrize("M", [1, 2, 7, 8, 9, 15, 16, 17, 40])
+def test_linear_matches_two_step_path_and_oracle(mid_case, M):
+    """w4a8_linear gives the very bits of w4a8_quantize_act followed by w4a8_gemm."""
+    case, layer = mid_case
+    y1 = _linear(case, layer, M)
+    qa, sa, asum = layer.quantize(case["x"][:M])
+    y2, _ = layer.gemm(qa, sa, asum)
+    assert np.array_equal(y1, y2)
+    r = cfast.w4a8_linear(case["x"][:M], case["qw"], case["sw"], case["z"], case["group"])
+    ok, ratio = onp.within_tolerance(y1, r["ref"])
+    assert ok, f"worst |err|/bound = {ratio:.3f}"
+
+
+def test_linear_edge_rows_and_many_slices():
+    """Zero rows, a saturating row, a subnormal scale, exact ties, on a layer whose K is split over
+    several slices with an uneven number of groups each."""
+    case = wl.make_layer(3072, 256, 41, 16)
+    rng = np.random.default_rng(9)
+    x = wl.bf16_bits_to_f32(case["x"]).copy()
+    x[0] = 0.0
+    x[1] *= np.float32(2.0 ** 100)
+    x[2] *= np.float32(2.0 ** -12)
+    x[3] *= np.float32(2.0 ** -40)
+    x[4] = np.arange(3072, dtype=np.float32) * np.float32(0.015625) - 8
+    x[5] = 1.0
+    x[6, :] = 0.0
+    x[6, 1500] = -5.0
+    case = dict(case, x=wl.f32_to_bf16_bits(x))
+    layer = DeviceLayer(case, 16)
+    for M in (7, 8, 16):
+        y1 = _linear(case, layer, M)
+        qa, sa, asum = layer.quantize(case["x"][:M])
+        y2, _ = layer.gemm(qa, sa, asum)
+        assert np.array_equal(y1, y2)
+        r = cfast.w4a8_linear(case["x"][:M], case["qw"], case["sw"], case["z"], case["group"])
+        finite = np.isfinite(r["ref"]).all(axis=1)
+        rms = float(np.sqrt(np.mean(r["ref"][finite] ** 2)))
+        ok, ratio = onp.within_tolerance(y1[finite], r["ref"][finite], rms_ref=rms)
+        assert ok, f"worst |err|/bound = {ratio:.3f}"
+
+
+def test_linear_full_size_spec_verify():
+    case = wl.make_config("spec_verify")
+    layer = DeviceLayer(case, case["M"])
+    y = _linear(case, layer, case["M"])
+    r = cfast.w4a8_linear(case["x"], case["qw"], case["sw"], case["z"], case["group"])
+    ok, ratio = onp.within_tolerance(y, r["ref"])
+    assert ok, f"worst |err|/bound = {ratio:.3f}"
+    for name in ("o", "gate_up", "down"):
+        c = wl.make_sweep_layer(name, 8)
+        lay = DeviceLayer(c, 8)
+        for M in (1, 4, 8):
+            yy = _linear(c, lay, M)
+            rr = cfast.w4a8_linear(c["x"][:M], c["qw"], c["sw"], c["z"], c["group"])
+            ok, ratio = onp.within_tolerance(yy, rr["ref"])
+            assert ok, f"{name} M={M}: worst |err|/bound = {ratio:.3f}"
+
+
+def test_linear_errors():
+    case, M = wl.make_config("tiny"), 4
+    layer = DeviceLayer(case, 16)
+    x = t_u16(case["x"][:M], torch.bfloat16)
+    with pytest.raises(B.W4A8Error) as e:
+        B.w4a8_linear(x, layer.packed, 100, layer.ws)
+    assert e.value.code == B.ERR_SHAPE
+    buf = torch.zeros(4 * 256 + 8, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.W4A8Error) as e:
+        B.w4a8_linear(buf[1:1 + 1024].view(4, 256), layer.packed, case["N"], layer.ws)
+    assert e.value.code == B.ERR_ALIGN
+    y = B.w4a8_linear(torch.empty((0, 256), dtype=torch.bfloat16, device="cuda"), layer.packed, case["N"], layer.ws)
+    assert y.shape == (0, case["N"])
