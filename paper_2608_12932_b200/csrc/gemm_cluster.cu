@@ -237,6 +237,27 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
 
     __syncwarp();
     ptx::cluster_wait();       // every CTA of the cluster has started: its shared memory may be written
+    if (S == 1) {
+        // a single slice owns the whole K range: its partials are the result, no exchange needed
+        if (warp < CL_ROW_WARPS) {
+            __nv_bfloat16* ycol = y + (size_t)ntile * TILE_N;
+#pragma unroll
+            for (int mb = 0; mb < MB; ++mb) {
+                const int m0 = 8 * mb + 2 * j;
+                if (m0 < M) {
+                    const float t = __half2float(__ushort_as_half(__ldcg(sa + m0)));
+                    ycol[(size_t)m0 * N + row_lo] = __float2bfloat16_rn(facc[mb][0] * t);
+                    ycol[(size_t)m0 * N + row_hi] = __float2bfloat16_rn(facc[mb][2] * t);
+                }
+                if (m0 + 1 < M) {
+                    const float t = __half2float(__ushort_as_half(__ldcg(sa + m0 + 1)));
+                    ycol[(size_t)(m0 + 1) * N + row_lo] = __float2bfloat16_rn(facc[mb][1] * t);
+                    ycol[(size_t)(m0 + 1) * N + row_hi] = __float2bfloat16_rn(facc[mb][3] * t);
+                }
+            }
+        }
+        return;
+    }
     if (warp < CL_ROW_WARPS) {
         // push this slice's partials to the CTAs that own them: slot `slice` of the owner's buffer
         const int T = M * TILE_N, chunk = (T + S - 1) / S;
