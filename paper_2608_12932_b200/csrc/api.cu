@@ -43,15 +43,15 @@ int device_sm_count() {
 
 // Between 17 and 64 tokens both kernel families are valid.  Measured on B200 (nanoseconds, cold
 // weights): the streaming kernel costs about 3000 + 950 x (blobs per SM) up to 32 tokens and, because
-// it then walks the token blocks twice, 7000 + 2030 x (blobs per SM) above; the tensor-core kernel
-// costs about 4000 + 440 x groups x (tiles per CTA) whatever the token count.  Pick the smaller estimate.
+// it then walks the token blocks twice, 7000 + 2030 x (blobs per SM) above; the tensor-core kernel's
+// estimate comes from its own planner (tile height, K split).  Pick the smaller estimate.
 bool small_m_prefers_tcgen05(int M, int N, int K, int sms) {
     if (M <= 16 || M > SPLITK_MAX_M) return M > SPLITK_MAX_M;
     const long G = K / GROUP, tiles = N / TILE_N;
     const long blobs_per_sm = (tiles * G) / sms;
     const long streaming_ns = M <= 32 ? 3000 + 950 * blobs_per_sm : 7000 + 2030 * blobs_per_sm;
-    const long tensor_ns = 4000 + 440 * G * ((tiles + sms - 1) / sms);
-    return tensor_ns < streaming_ns;
+    int tile_m = 0, split = 0;
+    return tcgen05_plan(M, N, K, sms, &tile_m, &split) < streaming_ns;
 }
 
 }  // namespace w4a8

@@ -38,6 +38,15 @@
 //   warp 2       producer of the packed blobs (1-D bulk copies)
 //   warps 4-7    unpack: raw blob -> signed int8 weight rows in TMEM
 //   warps 8-15   drain: tcgen05.ld -> convert -> FMA with the group scale; final bf16 store
+//
+// Split-K variant (SPLIT): when an [M, N] problem has fewer tiles than half the SMs, a tile is given
+// to a thread-block cluster of S CTAs, each walking G / S of the K groups (a CTA's time is close to
+// proportional to its number of groups, whatever the tile height).  The fp32 partials are reduced
+// like the small-M kernel's: after a cluster barrier (every CTA has finished its MMAs, so the
+// activation ring is free) each drain thread pushes its partials with st.shared::cluster into the
+// ring area of the CTA that owns that share of the tile (slot = pusher's rank), a second cluster
+// barrier, and the owner sums its S slots in rank order, applies the token scale and stores bf16.
+// (Pushing 16 bytes at a time into a channel-major buffer was measured slightly slower.)
 // Every wait is bounded; on expiry the CTA records W4A8_ERR_TIMEOUT, frees TMEM and exits.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -56,8 +65,10 @@ constexpr int NUM_UNPACK_WARPS = 4, NUM_DRAIN_WARPS = 8;
 constexpr int RAW_STRIDE = 8576;                 // BLOB_BYTES rounded up to a multiple of 128
 constexpr int A_COLS = GROUP / 4;                // 32 TMEM columns hold one group of a weight row (4 bytes per column)
 constexpr int TMEM_COLS = 512;
-// relative cost of one 208-, 128-, 64-token tile (same channels, same K), measured
-constexpr int TC_COST_208 = 148, TC_COST_128 = 123, TC_COST_64 = 100;
+// cost model of tcgen05_plan (nanoseconds, measured): per launch; per group of a 208-, 128-, 64-row tile; for splitting K
+// (cluster launch, two cluster barriers, exchange and reduction of a 208-, 128-, 64-row tile)
+constexpr long TC_FIXED_NS = 4000, TC_GROUP_NS[3] = {650, 540, 440}, TC_SPLIT_NS[3] = {10000, 7000, 4000};
+constexpr int TC_MAX_SPLIT = 4;
 
 // Shared-memory rings.  The activation tile comes from L2 through TMA with a latency of roughly
 // 2000 cycles, the packed blob from HBM likewise: both rings are deep enough to cover it.
@@ -97,19 +108,25 @@ __device__ __forceinline__ uint32_t sub_zero4(uint32_t q, uint32_t kz) {
     return (q + kz) ^ 0x80808080u;
 }
 
-template <int TILE_M, bool DEBUG>
+template <int TILE_M, bool DEBUG, bool SPLIT>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* __restrict__ packed,
                     const uint16_t* __restrict__ sa, __nv_bfloat16* __restrict__ y,
                     int32_t* __restrict__ debug_partials, uint32_t* __restrict__ status,
-                    int M, int N, int K, int m_tiles, int total_tiles) {
+                    int M, int N, int K, int m_tiles, int total_tiles, int S) {
     using C = Cfg<TILE_M>;
+    static_assert(!SPLIT || C::SB * C::B_BYTES >= TILE_M * TILE_N * 4 + 64, "the split-K exchange buffer lives in the activation ring");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-    const int G = K / GROUP;
+    const int GK = K / GROUP;                                   // groups of the whole K range (blob and output indexing)
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int unit = (int)blockIdx.x, num_units = (int)gridDim.x;
+    // SPLIT: a cluster of S CTAs per tile (one tile per cluster, no persistence); this CTA walks groups [g_lo, g_lo + G)
+    const int slice = SPLIT ? (int)ptx::cluster_ctarank() : 0;
+    const int unit = SPLIT ? (int)blockIdx.x / S : (int)blockIdx.x;
+    const int num_units = SPLIT ? (int)gridDim.x / S : (int)gridDim.x;
+    const int g_lo = SPLIT ? (int)(((long long)slice * GK) / S) : 0;
+    const int G = SPLIT ? (int)(((long long)(slice + 1) * GK) / S) - g_lo : GK;
 
     auto bar = [&](int i) { return smem_base + C::BAR_OFF + 8 * i; };
     // DONE[j % DONE_RING] completes its phase j / DONE_RING when the MMAs of pipeline step j have finished: that
@@ -151,6 +168,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
         mtile = t % m_tiles;
     };
 
+    bool exchanged = false;                     // SPLIT: this thread has passed the first cluster barrier
     if (warp < 4) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         // A producer iteration is a chain of dependent round trips (barrier probe, expect-tx, copy
@@ -168,7 +186,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                     const uint32_t sb = it % C::SB;
                     if (it >= (uint32_t)C::SB && !(ok = ptx::mbar_wait(done_bar(it - C::SB), done_parity(it - C::SB), abort_flag))) break;
                     ptx::mbar_arrive_expect_tx(bar(B_FULL + sb), C::B_BYTES);
-                    ptx::tma_load_2d(smem_base + C::B_OFF + sb * C::B_BYTES, &tmap_qa, g * GROUP, mtile * TILE_M,
+                    ptx::tma_load_2d(smem_base + C::B_OFF + sb * C::B_BYTES, &tmap_qa, (g_lo + g) * GROUP, mtile * TILE_M,
                                      bar(B_FULL + sb));
                 }
             }
@@ -183,7 +201,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
             for (int tile = unit; tile < total_tiles && ok; tile += num_units) {
                 int ntile, mtile;
                 tile_of(tile, ntile, mtile);
-                const uint8_t* src = packed + (size_t)ntile * G * BLOB_BYTES;
+                const uint8_t* src = packed + ((size_t)ntile * GK + g_lo) * BLOB_BYTES;
                 for (int g = 0; g < G; ++g, ++it) {
                     if ((int)(it % PRODUCER_LANES) != lane) continue;
                     const uint32_t sr = it % C::SR, pr = (it / C::SR) & 1;
@@ -293,7 +311,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
             tile_of(tile, ntile, mtile);
             const int n = ntile * TILE_N + n_local;
             const int m_base = mtile * TILE_M + h * C::W;
-            const uint8_t* sw_ptr = packed + (size_t)ntile * G * BLOB_BYTES + BLOB_SCALE_OFF + 2 * n_local;
+            const uint8_t* sw_ptr = packed + ((size_t)ntile * GK + g_lo) * BLOB_BYTES + BLOB_SCALE_OFF + 2 * n_local;
             float facc[C::W];
 #pragma unroll
             for (int i = 0; i < C::W; ++i) facc[i] = 0.0f;
@@ -333,13 +351,29 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                             facc[ch * 32 + i] = fmaf(sw, (float)di, facc[ch * 32 + i]);     // exact convert: |D| < 2^24
                             if (DEBUG) {
                                 const int m = m_base + ch * 32 + i;
-                                if (m < M) debug_partials[((size_t)m * G + g) * N + n] = di;
+                                if (m < M) debug_partials[((size_t)m * GK + g_lo + g) * N + n] = di;
                             }
                         }
                     }
                 }
             }
             if (!ok) break;
+            if (SPLIT) {
+                // every CTA of the cluster is past its last MMA: the activation rings are free and become
+                // the exchange buffers; push this thread's partials to the CTAs that own them
+                ptx::cluster_sync();
+                exchanged = true;
+                // element (token t, channel n) of the tile has index t * 128 + n; the indices are dealt out to
+                // the S CTAs in contiguous chunks
+                const int chunk = (TILE_M * TILE_N + S - 1) / S;
+                const uint32_t red = smem_base + C::B_OFF;
+#pragma unroll
+                for (int i = 0; i < C::W; ++i) {
+                    const int idx = (h * C::W + i) * TILE_N + n_local, owner = idx / chunk;
+                    ptx::st_dsmem_f32(ptx::map_to_cta(red + (uint32_t)(slice * chunk + idx - owner * chunk) * 4u, (uint32_t)owner), facc[i]);
+                }
+                break;                          // one tile per cluster
+            }
             // Epilogue: token scale, bf16, and a transpose through shared memory so that global
             // stores are 16 bytes per lane along the channel dimension (a thread owns a channel,
             // the output is token-major).  Blocks of up to 32 tokens x this warp's 32 channels.
@@ -366,6 +400,29 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
         }
     }
 
+    if (SPLIT) {
+        // first barrier for every thread that has not passed it in the drain role, then the second one
+        // (release after the pushes, acquire before the sums); this CTA then reduces its share of the tile
+        if (!exchanged) ptx::cluster_sync();
+        ptx::cluster_sync();
+        if (unit < total_tiles && !*abort_flag) {
+            int ntile, mtile;
+            tile_of(unit, ntile, mtile);
+            const int chunk = (TILE_M * TILE_N + S - 1) / S;
+            const int lo = slice * chunk;
+            const int cnt = (TILE_M * TILE_N - lo) < chunk ? (TILE_M * TILE_N - lo) : chunk;
+            const float* red = reinterpret_cast<const float*>(smem + C::B_OFF);
+            for (int i = tid; i < cnt; i += TC_THREADS) {
+                float acc = 0.0f;
+                for (int s2 = 0; s2 < S; ++s2) acc += red[s2 * chunk + i];        // rank order: deterministic
+                const int idx = lo + i, m = mtile * TILE_M + idx / TILE_N, nn = idx % TILE_N;
+                if (m < M) {
+                    const float t = __half2float(__ushort_as_half(__ldg(sa + m)));
+                    y[(size_t)m * N + (size_t)ntile * TILE_N + nn] = __float2bfloat16_rn(acc * t);
+                }
+            }
+        }
+    }
     if (*abort_flag && lane == 0) atomicExch(status, (uint32_t)W4A8_ERR_TIMEOUT);
     ptx::tc_fence_before_sync();
     __syncthreads();
@@ -375,8 +432,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
     }
 }
 
-template <int TILE_M, bool DEBUG>
-cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed, void* y, int M, int N, int K,
+template <int TILE_M, bool DEBUG, bool SPLIT>
+cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed, void* y, int M, int N, int K, int S,
                         void* workspace, int32_t* debug_partials, cudaStream_t stream) {
     using C = Cfg<TILE_M>;
     CUtensorMap tmap;
@@ -390,58 +447,115 @@ cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     const int sms = device_sm_count();
     if (!attr_done[dev]) {
-        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<TILE_M, DEBUG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  C::SMEM_ALLOC);
         if (e != cudaSuccess) return e;
         attr_done[dev] = true;
     }
     const int m_tiles = (M + TILE_M - 1) / TILE_M;
     const int total = m_tiles * (N / TILE_N);
-    const int grid = total < sms ? total : sms;
+    // persistent: at most one CTA per SM; split-K: one cluster of S CTAs per tile
+    const int grid = SPLIT ? total * S : (total < sms ? total : sms);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    gemm_tcgen05_kernel<TILE_M, DEBUG><<<grid, TC_THREADS, C::SMEM_ALLOC, stream>>>(
-        tmap, static_cast<const uint8_t*>(packed), sa, static_cast<__nv_bfloat16*>(y), debug_partials,
-        reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF), M, N, K, m_tiles, total);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(TC_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = C::SMEM_ALLOC;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = SPLIT ? (unsigned)S : 1u;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT>, tmap, static_cast<const uint8_t*>(packed), sa,
+                              static_cast<__nv_bfloat16*>(y), debug_partials, reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF),
+                              M, N, K, m_tiles, total, S);
+}
+
+// Clusters of S CTAs of the split-K kernel that the device can hold at once (S CTAs need S free SMs
+// of one GPC, so this is less than SMs / S); 0 if the query fails.  Cached per device.
+template <int TILE_M>
+int max_active_clusters(int S) {
+    static int cached[64][TC_MAX_SPLIT + 1] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || S < 2 || S > TC_MAX_SPLIT) return 0;
+    if (cached[dev][S] == 0) {
+        using C = Cfg<TILE_M>;
+        int n = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(S * 64), 1, 1);
+        cfg.blockDim = dim3(TC_THREADS, 1, 1);
+        cfg.dynamicSmemBytes = C::SMEM_ALLOC;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = (unsigned)S;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        if (cudaFuncSetAttribute(gemm_tcgen05_kernel<TILE_M, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 C::SMEM_ALLOC) != cudaSuccess ||
+            cudaOccupancyMaxActiveClusters(&n, gemm_tcgen05_kernel<TILE_M, false, true>, &cfg) != cudaSuccess)
+            n = -1;
+        cached[dev][S] = n > 0 ? n : -1;
+    }
+    return cached[dev][S] > 0 ? cached[dev][S] : 0;
 }
 
 template <bool DEBUG>
-cudaError_t launch_height(int tile_m, const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
-                          int M, int N, int K, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
-    if (tile_m == 64) return launch_tile<64, DEBUG>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
-    if (tile_m == 128) return launch_tile<128, DEBUG>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
-    return launch_tile<208, DEBUG>(qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+cudaError_t launch_plan(int tile_m, int S, const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
+                        int M, int N, int K, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
+    if (S > 1) {
+        if (tile_m == 64) return launch_tile<64, DEBUG, true>(qa, sa, packed, y, M, N, K, S, workspace, debug_partials, stream);
+        if (tile_m == 128) return launch_tile<128, DEBUG, true>(qa, sa, packed, y, M, N, K, S, workspace, debug_partials, stream);
+        return launch_tile<208, DEBUG, true>(qa, sa, packed, y, M, N, K, S, workspace, debug_partials, stream);
+    }
+    if (tile_m == 64) return launch_tile<64, DEBUG, false>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
+    if (tile_m == 128) return launch_tile<128, DEBUG, false>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
+    return launch_tile<208, DEBUG, false>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
 }
 
 }  // namespace
 
-// Token-tile height for an [M, N] problem.  A CTA's time per tile has a part that does not depend on
-// the tile height (unpacking the tile's weights) and a part that does (MMAs, drain, activation
-// traffic); COST holds the measured ratio.  The persistent grid runs ceil(tiles / SMs) tiles per
-// CTA, so the height with the smallest (tiles per CTA) x (cost per tile) wins: tall tiles when
-// there are several waves of them, short ones when a tall tiling would leave SMs idle.
-int tcgen05_tile_m(int M, int N, int sms) {
+// Tile height and K split for an [M, N, K] problem, from a cost model fitted to measurements on B200:
+// a CTA spends about TC_FIXED_NS on launch, set-up and pipeline fill, then TC_GROUP_NS[height] per
+// 128-k group of every tile it walks (the weight unpack, whose cost does not depend on the height,
+// dominates a group, so taller tiles are cheaper per token); a K split into S slices costs
+// TC_SPLIT_NS for the cluster exchange.  Tall tiles win when there are several waves of them, short
+// ones when a tall tiling would leave SMs idle, and a K split when even the shortest tiling does.
+long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split) {
     const int heights[3] = {208, 128, 64};
-    const int cost[3] = {TC_COST_208, TC_COST_128, TC_COST_64};
-    const int n_tiles = N / TILE_N;
-    int best = 64;
-    long best_cost = -1;
+    const int n_tiles = N / TILE_N, G = K / GROUP;
+    long best_ns = -1;
+    *tile_m = 64;
+    *split = 1;
     for (int i = 0; i < 3; ++i) {
         if (heights[i] > 64 && M <= heights[i + 1]) continue;        // the next height down already covers M in one tile
         const long tiles = (long)((M + heights[i] - 1) / heights[i]) * n_tiles;
-        const long c = ((tiles + sms - 1) / sms) * cost[i];
-        if (best_cost < 0 || c < best_cost) { best_cost = c; best = heights[i]; }   // ties go to the taller tile
+        const long waves = (tiles + sms - 1) / sms;
+        for (int S = 1; S <= TC_MAX_SPLIT; ++S) {
+            if (S > 1) {
+                if (tiles * S > sms || G / S < 4) break;
+                const int room = i == 0 ? max_active_clusters<208>(S) : (i == 1 ? max_active_clusters<128>(S) : max_active_clusters<64>(S));
+                if (tiles > room) continue;                          // the clusters must all be resident at once
+            }
+            const long ns = TC_FIXED_NS + waves * TC_GROUP_NS[i] * ((G + S - 1) / S) + (S > 1 ? TC_SPLIT_NS[i] : 0);
+            if (best_ns < 0 || ns < best_ns) { best_ns = ns; *tile_m = heights[i]; *split = S; }   // ties: taller tile, fewer slices
+        }
     }
-    return best;
+    return best_ns;                                                   // the estimate, for the caller's choice of kernel family
 }
 
 cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
                                 int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream) {
-    const int tile_m = tcgen05_tile_m(M, N, device_sm_count());
+    int tile_m = 64, S = 1;
+    tcgen05_plan(M, N, K, device_sm_count(), &tile_m, &S);
     if (debug_partials)
-        return launch_height<true>(tile_m, qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
-    return launch_height<false>(tile_m, qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+        return launch_plan<true>(tile_m, S, qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+    return launch_plan<false>(tile_m, S, qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
 }
 
 }  // namespace w4a8

@@ -57,7 +57,7 @@ cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int3
 cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
                                 int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream);
-int tcgen05_tile_m(int M, int N, int sms);    // token-tile height the tcgen05 launcher picks
+long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split);    // tile height and K split the tcgen05 launcher picks; returns its time estimate (ns)
 bool small_m_prefers_tcgen05(int M, int N, int K, int sms);
 
 }  // namespace w4a8

@@ -128,6 +128,20 @@ def test_long_k_many_slices():
     check_case(case, layer, 70, "tcgen05")
 
 
+def test_tcgen05_k_split_uneven_slices():
+    """Few tiles, so the tensor-core kernel splits K over a cluster: 13 groups over 2 or 3 slices
+    (uneven shares), 24 groups over 4; debug partials from every slice land at their own group index."""
+    case = wl.make_layer(1664, 256, 37, 210)          # G = 13, two channel tiles
+    layer = DeviceLayer(case, 210)
+    for M in (33, 64, 100, 128, 129, 210):
+        check_case(case, layer, M, "tcgen05")
+    case = wl.make_layer(3072, 384, 38, 64)           # G = 24, three channel tiles
+    layer = DeviceLayer(case, 64)
+    for M in (17, 64):
+        check_case(case, layer, M, "tcgen05")
+        check_case(case, layer, M, "auto", debug=False)
+
+
 def test_ring_reuse_many_groups_per_cta():
     """Wide layer, few slices: each CTA walks more groups than its ring has stages."""
     case = wl.make_layer(4096, 4096, 34, 24)         # 32 tiles -> 8 slices of 4 groups; and
