@@ -360,16 +360,22 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
 
 // Slices per tile for the cluster kernel, at most 8 (portable cluster size) and never more than
 // the number of groups.  Measured on the four layer shapes: one m-block (M <= 8) runs best with
-// about 1.4 CTAs per SM (two co-resident CTAs per SM leave room for the next launch to prefetch),
-// larger M, whose CTAs hold more registers and shared memory, with about 0.75.
+// about 1.4 CTAs per SM (two co-resident CTAs per SM leave room for the next launch to prefetch);
+// larger M, whose CTAs hold more registers and shared memory, with the largest power of two that
+// keeps the launch within 0.9 CTAs per SM (clusters of 3 were always slower than 2 or 4).
 int cluster_num_slices(int M, int N, int K) {
     const int G = K / GROUP, tiles = N / TILE_N, sms = device_sm_count();
     if (const char* e = getenv("W4A8_CLUSTER_S")) {      // tuning aid: force the slice count
         int v = atoi(e);
         if (v >= 1 && v <= CL_MAX_S && v <= G) return v;
     }
-    const int target = M <= 8 ? (sms * 14) / 10 : (sms * 3) / 4;
-    int s = (target + tiles / 2) / tiles;
+    int s;
+    if (M <= 8) {
+        s = ((sms * 14) / 10 + tiles / 2) / tiles;
+    } else {
+        s = 1;
+        while (2 * s <= CL_MAX_S && tiles * 2 * s <= (sms * 9) / 10) s *= 2;
+    }
     if (s > CL_MAX_S) s = CL_MAX_S;
     if (s > G) s = G;
     if (s < 1) s = 1;
