@@ -15,9 +15,11 @@
 // overwrites its buffer, so a buffer needs no preparation: the drain hands it back as soon as
 // its columns are in registers.
 //
-// What bounds this kernel is shared-memory bandwidth (about 128 B/clk per SM, shared by the
-// tensor core's operand reads, the bulk-copy fills and ordinary loads/stores) and the TMEM
-// read port, not the tensor pipe.  Hence:
+// The tensor pipe is not what bounds this kernel (it is busy under a third of the time): the CUDA
+// cores must take every accumulator element out of TMEM after every group and spend two
+// instructions on it, the unpack shares the integer pipe with that conversion, and shared memory
+// (about 128 B/clk per SM) is shared by the tensor core's operand reads, the bulk-copy fills and
+// ordinary loads.  Design choices made on measurements:
 //  * the unpacked weights never touch shared memory: an unpack thread owns one weight row
 //    (= one TMEM lane), converts its 64 packed bytes in registers and writes the 128 signed
 //    bytes to 32 TMEM columns with tcgen05.st; the MMA takes its A operand from TMEM.  That
@@ -25,8 +27,13 @@
 //  * the token tile is 208 rows, not 256: two accumulator buffers of 208 columns plus three
 //    32-column weight stages fill the 512 TMEM columns exactly, and M = 1024 or 4096 splits
 //    into 208-row tiles with 1.5 % padding;
-//  * there is no accumulator bias / re-arm: tcgen05.st traffic to TMEM is as expensive as
-//    tcgen05.ld traffic, and the int->float conversion runs on a pipe the FMAs do not use.
+//  * there is no accumulator bias / re-arm (which would turn the int->float conversion into an
+//    FMA-pipe add): tcgen05.st traffic to TMEM costs as much port time as tcgen05.ld traffic, more
+//    than the conversion;
+//  * two threads issue the MMAs, one for the even and one for the odd steps: a step costs its issuer
+//    three barrier probes, four MMAs and a commit, each a round trip of about a hundred cycles;
+//  * one tcgen05.commit per step, on a ring of "step done" barriers, frees the step's weight and
+//    activation stages and publishes its accumulator.
 //
 // Zero points are subtracted while unpacking (weights become signed, -15..15), so the int32
 // accumulator is directly D = sum (q_w - z) q_a; identical to P - z*sum(q_a), and it moves the
@@ -59,7 +66,6 @@ namespace {
 
 constexpr int TC_THREADS = 512;
 constexpr int WARP_PRODUCER = 0, WARP_MMA = 1, WARP_RAW_PRODUCER = 2, WARP_MMA_ODD = 3, WARP_UNPACK0 = 4, WARP_DRAIN0 = 8;
-constexpr int PRODUCER_LANES = 4;                // threads per copy producer
 constexpr int DONE_RING = 8;                     // "group finished" barriers; every role stays within 8 groups of the others
 constexpr int NUM_UNPACK_WARPS = 4, NUM_DRAIN_WARPS = 8;
 constexpr int RAW_STRIDE = 8576;                 // BLOB_BYTES rounded up to a multiple of 128
@@ -171,10 +177,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
     bool exchanged = false;                     // SPLIT: this thread has passed the first cluster barrier
     if (warp < 4) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
-        // A producer iteration is a chain of dependent round trips (barrier probe, expect-tx, copy
-        // issue) of several hundred cycles; PRODUCER_LANES lanes take the pipeline steps round-robin so
-        // that the chains overlap.
-        if (warp == WARP_PRODUCER && lane < PRODUCER_LANES) {
+        if (warp == WARP_PRODUCER && lane == 0) {
             // ------------------------------------------------ producer: activation tiles ----
             uint32_t it = 0;
             bool ok = true;
@@ -182,7 +185,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 int ntile, mtile;
                 tile_of(tile, ntile, mtile);
                 for (int g = 0; g < G; ++g, ++it) {
-                    if ((int)(it % PRODUCER_LANES) != lane) continue;
                     const uint32_t sb = it % C::SB;
                     if (it >= (uint32_t)C::SB && !(ok = ptx::mbar_wait(done_bar(it - C::SB), done_parity(it - C::SB), abort_flag))) break;
                     ptx::mbar_arrive_expect_tx(bar(B_FULL + sb), C::B_BYTES);
@@ -194,7 +196,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 const uint64_t t0 = ptx::globaltimer_ns();
                 while (ptx::globaltimer_ns() - t0 < 200000ull) {}
             }
-        } else if (warp == WARP_RAW_PRODUCER && lane < PRODUCER_LANES) {
+        } else if (warp == WARP_RAW_PRODUCER && lane == 0) {
             // --------------------------------------------------- producer: packed blobs ----
             uint32_t it = 0;
             bool ok = true;
@@ -203,7 +205,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 tile_of(tile, ntile, mtile);
                 const uint8_t* src = packed + ((size_t)ntile * GK + g_lo) * BLOB_BYTES;
                 for (int g = 0; g < G; ++g, ++it) {
-                    if ((int)(it % PRODUCER_LANES) != lane) continue;
                     const uint32_t sr = it % C::SR, pr = (it / C::SR) & 1;
                     if (!(ok = ptx::mbar_wait(bar(RAW_EMPTY + sr), pr ^ 1, abort_flag))) break;
                     ptx::mbar_arrive_expect_tx(bar(RAW_FULL + sr), BLOB_BYTES);
