@@ -62,8 +62,11 @@ __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, 
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-template <int MB>
-__global__ void __launch_bounds__(CL_THREADS)
+// MINB = 2 caps the registers so that two CTAs fit on an SM: wanted when a launch has more CTAs than
+// SMs anyway (they then share SMs instead of queueing); with fewer CTAs than SMs it only invites the
+// cluster scheduler to pack two of them onto one SM and leave others idle.
+template <int MB, int MINB>
+__global__ void __launch_bounds__(CL_THREADS, MINB)
 gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t* __restrict__ sa,
                     const int32_t* __restrict__ asum, const uint8_t* __restrict__ packed,
                     __nv_bfloat16* __restrict__ y, int M, int N, int K, int S, int ng_max, int stages,
@@ -295,7 +298,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
     }
 }
 
-template <int MB>
+template <int MB, int MINB>
 cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed, void* y,
                       int M, int N, int K, int S, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
     const int G = K / GROUP;
@@ -327,7 +330,7 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     static bool attr_done[64] = {false};
     if (!attr_done[dev]) {
-        e = cudaFuncSetAttribute(gemm_cluster_kernel<MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        e = cudaFuncSetAttribute(gemm_cluster_kernel<MB, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         attr_done[dev] = true;
     }
@@ -352,7 +355,7 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
     cfg.attrs = attrs;
     cfg.numAttrs = 3;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    return cudaLaunchKernelEx(&cfg, gemm_cluster_kernel<MB>, tmap, sa, asum, static_cast<const uint8_t*>(packed),
+    return cudaLaunchKernelEx(&cfg, gemm_cluster_kernel<MB, MINB>, tmap, sa, asum, static_cast<const uint8_t*>(packed),
                               static_cast<__nv_bfloat16*>(y), M, N, K, S, ng_max, stages,
                               reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF), debug_partials);
 }
@@ -386,10 +389,14 @@ cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int3
                                 void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream) {
     const int S = cluster_num_slices(M, N, K);
-    if (M <= 8) return launch_mb<1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
-    if (M <= 16) return launch_mb<2>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
-    if (M <= 32) return launch_mb<4>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
-    return launch_mb<8>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+    if (M <= 8) return launch_mb<1, 2>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);   // two launches co-resident
+    if (M <= 16) {
+        if ((N / TILE_N) * S > device_sm_count())
+            return launch_mb<2, 2>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+        return launch_mb<2, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+    }
+    if (M <= 32) return launch_mb<4, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+    return launch_mb<8, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
 }
 
 }  // namespace w4a8
