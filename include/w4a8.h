@@ -108,7 +108,8 @@ w4a8_status w4a8_quantize_act(const void* x_bf16, int M, int K, int group,
  *   y_bf16           [M,N] row-major bf16
  *   workspace        >= w4a8_workspace_bytes(M,N,K,group) bytes, 256-byte aligned, header zeroed once
  *   debug_partials   NULL, or [M,K/group,N] int32 that receives D (slower debug mode)
- * Dispatch: M <= 64 runs the split-K weight-streaming kernel, larger M the tcgen05 kernel.
+ * Dispatch: up to 16 tokens the split-K weight-streaming kernel, above 64 the tcgen05 kernel, in
+ * between whichever a measured cost model predicts faster for the shape (w4a8_plan tells which).
  * Results are run-to-run deterministic.  The kernels are launched with programmatic stream
  * serialisation: when consecutive library calls share a stream, a kernel may start (and prefetch
  * weights) before its predecessor has finished, and waits on the device before it reads any
@@ -119,6 +120,20 @@ w4a8_status w4a8_gemm(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
                       int M, int N, int K, int group,
                       void* workspace, size_t workspace_bytes,
                       int32_t* debug_partials, void* stream);
+
+/*
+ * What w4a8_gemm would launch for a problem size on the current device (host-only query, nothing is
+ * enqueued): the kernel family, and for W4A8_PATH_SPLITK the number of K slices per 128-channel tile
+ * (cluster size), for W4A8_PATH_TCGEN05 the token-tile height (64, 128 or 208) and the number of K
+ * slices (1 = no split).  Any output pointer may be NULL.  W4A8_ERR_SHAPE for an unsupported shape.
+ */
+typedef struct {
+    w4a8_path family;   /* W4A8_PATH_SPLITK or W4A8_PATH_TCGEN05 */
+    int tile_m;         /* tcgen05: token rows per tile; split-K: 8 x token blocks per CTA (8, 16, 32 or 64) */
+    int k_slices;       /* CTAs that share the K range of one tile */
+    int ctas;           /* CTAs of the launch */
+} w4a8_plan_info;
+w4a8_status w4a8_plan(int M, int N, int K, int group, w4a8_plan_info* out);
 
 /* w4a8_gemm with the kernel family forced (path-consistency tests, benchmarking). */
 w4a8_status w4a8_gemm_path(w4a8_path path,

@@ -19,7 +19,7 @@ WORKSPACE_HEADER_BYTES = 4096
 
 EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w4a8_workspace_init",
            "w4a8_pack_weights", "w4a8_unpack_weights", "w4a8_quantize_act", "w4a8_gemm", "w4a8_gemm_path",
-           "w4a8_linear", "w4a8_linear_host", "w4a8_gemm_static_scratch", "w4a8_check_status")
+           "w4a8_linear", "w4a8_linear_host", "w4a8_gemm_static_scratch", "w4a8_check_status", "w4a8_plan")
 
 _lib = None
 
@@ -57,6 +57,8 @@ def lib():
         L.w4a8_gemm.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp, vp]
         L.w4a8_gemm_path.restype = ci
         L.w4a8_gemm_path.argtypes = [ci, vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp, vp]
+        L.w4a8_plan.restype = ci
+        L.w4a8_plan.argtypes = [ci, ci, ci, ci, vp]
         L.w4a8_linear.restype = ci
         L.w4a8_linear.argtypes = [vp, vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, sz, vp]
         L.w4a8_linear_host.restype = ci
@@ -172,6 +174,17 @@ def w4a8_gemm(qa, sa, asum, packed_w, N, workspace, group=GROUP, out=None, debug
                                     _ptr(workspace), workspace.numel(), _ptr(debug_partials), _stream(stream))
     _check(code, "w4a8_gemm")
     return out
+
+
+class PlanInfo(ctypes.Structure):
+    _fields_ = [("family", ctypes.c_int), ("tile_m", ctypes.c_int), ("k_slices", ctypes.c_int), ("ctas", ctypes.c_int)]
+
+
+def w4a8_plan(M, N, K, group=GROUP):
+    """What w4a8_gemm would launch for this size on the current device: dict(family, tile_m, k_slices, ctas)."""
+    info = PlanInfo()
+    _check(lib().w4a8_plan(M, N, K, group, ctypes.byref(info)), "w4a8_plan")
+    return {"family": info.family, "tile_m": info.tile_m, "k_slices": info.k_slices, "ctas": info.ctas}
 
 
 def w4a8_linear(x, packed_w, N, workspace, group=GROUP, out=None, scratch=None, stream=None):

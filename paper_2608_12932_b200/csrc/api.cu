@@ -166,6 +166,25 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
     return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
 
+w4a8_status w4a8_plan(int M, int N, int K, int group, w4a8_plan_info* out) {
+    if (!shape_ok(N, K, group) || M <= 0) return W4A8_ERR_SHAPE;
+    const int sms = device_sm_count(), tiles = N / TILE_N;
+    w4a8_plan_info p;
+    if (!small_m_prefers_tcgen05(M, N, K, sms)) {
+        p.family = W4A8_PATH_SPLITK;
+        p.tile_m = M <= 8 ? 8 : (M <= 16 ? 16 : (M <= 32 ? 32 : 64));
+        p.k_slices = cluster_num_slices(M, N, K);
+        p.ctas = tiles * p.k_slices;
+    } else {
+        p.family = W4A8_PATH_TCGEN05;
+        tcgen05_plan(M, N, K, sms, &p.tile_m, &p.k_slices);
+        const int all = ((M + p.tile_m - 1) / p.tile_m) * tiles;
+        p.ctas = p.k_slices > 1 ? all * p.k_slices : (all < sms ? all : sms);
+    }
+    if (out) *out = p;
+    return W4A8_OK;
+}
+
 w4a8_status w4a8_gemm(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
                       const void* packed_w, void* y_bf16,
                       int M, int N, int K, int group,

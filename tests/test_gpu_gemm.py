@@ -371,3 +371,15 @@ def test_linear_errors():
     assert e.value.code == B.ERR_ALIGN
     y = B.w4a8_linear(torch.empty((0, 256), dtype=torch.bfloat16, device="cuda"), layer.packed, case["N"], layer.ws)
     assert y.shape == (0, case["N"])
+
+
+def test_plan_matches_the_device():
+    """On the GPU the planner may split K over a cluster when a problem has few tiles; whatever it
+    picks fits the machine, and the result of the dispatch it describes is right."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    p = B.w4a8_plan(64, 4096, 12288)                  # down projection, 32 tiles, 96 groups
+    assert p["family"] == B.PATH_TCGEN05 and p["k_slices"] > 1 and p["ctas"] <= sms
+    p = B.w4a8_plan(8, 6144, 4096)
+    assert p["family"] == B.PATH_SPLITK and p["ctas"] == 48 * p["k_slices"]
+    p = B.w4a8_plan(1024, 24576, 4096)
+    assert p == {"family": B.PATH_TCGEN05, "tile_m": 208, "k_slices": 1, "ctas": sms}

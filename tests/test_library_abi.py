@@ -54,6 +54,40 @@ def test_size_queries():
     assert B.w4a8_packed_bytes(128 * 961, 128) == 0          # more tiles than the workspace header has counters
 
 
+def test_plan_query_invariants():
+    """w4a8_plan is host-only: on a machine without a GPU it assumes 148 SMs and no cluster occupancy
+    (so no K split of the tensor-core kernel), and its answers obey the dispatch rules."""
+    sms = 148
+    for (K, N) in list(wl.LAYERS.values()) + [(256, 256), (1024, 384), (3072, 256)]:
+        tiles, G = N // 128, K // 128
+        for M in (1, 7, 8, 9, 16, 17, 32, 33, 64, 65, 128, 200, 256, 512, 1024, 4096):
+            p = B.w4a8_plan(M, N, K)
+            assert p["family"] in (B.PATH_SPLITK, B.PATH_TCGEN05)
+            if M <= 16:
+                assert p["family"] == B.PATH_SPLITK
+            if M > 64:
+                assert p["family"] == B.PATH_TCGEN05
+            if p["family"] == B.PATH_SPLITK:
+                assert p["tile_m"] in (8, 16, 32, 64) and p["tile_m"] >= min(M, 64)
+                assert 1 <= p["k_slices"] <= min(8, G) and p["ctas"] == tiles * p["k_slices"]
+            else:
+                assert p["tile_m"] in (64, 128, 208) and 1 <= p["k_slices"] <= 4
+                all_tiles = -(-M // p["tile_m"]) * tiles
+                if p["k_slices"] > 1:
+                    assert p["ctas"] == all_tiles * p["k_slices"] <= sms and G // p["k_slices"] >= 4
+                else:
+                    assert p["ctas"] == min(all_tiles, sms)
+                # never a taller tile than the next height down that already covers M
+                assert not (p["tile_m"] == 208 and M <= 128) and not (p["tile_m"] == 128 and M <= 64)
+    # several waves of tiles: the tallest tile; a bad shape: an error
+    assert B.w4a8_plan(4096, 24576, 4096)["tile_m"] == 208
+    with pytest.raises(B.W4A8Error) as e:
+        B.w4a8_plan(8, 100, 256)
+    assert e.value.code == B.ERR_SHAPE
+    with pytest.raises(B.W4A8Error):
+        B.w4a8_plan(0, 256, 256)
+
+
 def test_status_strings():
     seen = {B.status_string(c) for c in range(8)}
     assert len(seen) == 8 and "ok" in seen
