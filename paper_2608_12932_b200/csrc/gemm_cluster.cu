@@ -14,10 +14,12 @@
 //    D = P - z * sum(q_a) with the group sums from the quantise kernel; fp32 group scales; the odd
 //    set's partial sums are added to the even set's through shared memory (fixed order).
 //  * reduction: the tile's M x 128 outputs are split into S contiguous shares, one per CTA of the
-//    cluster.  Every CTA pushes each of its fp32 partials into the owner's shared memory (slot =
-//    pusher's rank) with st.shared::cluster, then one cluster barrier (release/acquire); the owner
-//    sums its S slots in rank order (fixed order: deterministic), applies the token scale and
-//    stores bf16.  After the barrier a CTA reads only its own shared memory, so it may exit freely.
+//    cluster.  A CTA lays its fp32 partials out as [token][channel] in its own shared memory and
+//    pushes them in 16-byte pieces into the owners' shared memory (slot = pusher's rank) with
+//    st.shared::cluster (one store instruction of a warp then goes to one owner), then one cluster
+//    barrier (release/acquire); the owner sums its S slots in rank order (fixed order:
+//    deterministic), applies the token scale and stores bf16.  After the barrier a CTA reads only
+//    its own shared memory, so it may exit freely.
 //  * sizing: the number of slices minimises ceil(CTAs / SMs) * ceil(G / S); a launch that fits in
 //    one wave keeps its CTAs under half an SM's shared memory and prefetches as much of its slice
 //    as fits, so that two consecutive launches can be resident together and the weight stream of
@@ -48,8 +50,8 @@ __host__ __device__ inline ClLayout cl_layout(int mb, int stages, int ng_max) {
     L.bar_off = L.blob_off + stages * CL_BLOB_STRIDE;
     L.asum_off = L.bar_off + 2 * CL_MAX_STAGES * 8;
     L.red_off = (L.asum_off + 8 * mb * ng_max * 4 + 15) & ~15;
-    L.set_off = L.red_off + (8 * mb * TILE_N + CL_MAX_S) * 4;     // S slots x ceil(M*128/S) floats
-    L.misc_off = L.set_off + CL_ROW_WARPS * 32 * 4 * mb * 4;      // odd set's partials: 4*mb floats per thread
+    L.set_off = L.red_off + (8 * mb * (TILE_N / 4) + CL_MAX_S) * 16;   // S slots x ceil(M*32/S) float4
+    L.misc_off = L.set_off + 8 * mb * TILE_N * 4;                 // this CTA's partial sums, [token][channel] fp32
     L.total = L.misc_off + 16;
     return L;
 }
@@ -220,19 +222,28 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
             for (int st = 0; st < stages; ++st)
                 for (int spin = 0; spin < (1 << 16) && !ptx::mbar_try_wait(full_bar(st), 0); ++spin) {}
         }
-        // odd-group partials join the even-group ones (even + odd: fixed order)
-        float* set_buf = reinterpret_cast<float*>(smem + L.set_off) + ((warp & 7) * 32 + lane) * 4 * MB;
+        // odd-group partials join the even-group ones (even + odd: fixed order) in a [token][channel]
+        // buffer, from which the exchange below pushes 16-byte pieces
+        float* part = reinterpret_cast<float*>(smem + L.set_off);
         if (set == 1) {
 #pragma unroll
-            for (int mb = 0; mb < MB; ++mb)
-                *reinterpret_cast<float4*>(set_buf + 4 * mb) = make_float4(facc[mb][0], facc[mb][1], facc[mb][2], facc[mb][3]);
+            for (int mb = 0; mb < MB; ++mb) {
+                float* p = part + (8 * mb + 2 * j) * TILE_N;
+                p[row_lo] = facc[mb][0]; p[TILE_N + row_lo] = facc[mb][1];
+                p[row_hi] = facc[mb][2]; p[TILE_N + row_hi] = facc[mb][3];
+            }
         }
         ptx::named_bar_sync(1, CL_CONSUMER_WARPS * 32);
         if (set == 0) {
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb) {
-                const float4 o = *reinterpret_cast<const float4*>(set_buf + 4 * mb);
-                facc[mb][0] += o.x; facc[mb][1] += o.y; facc[mb][2] += o.z; facc[mb][3] += o.w;
+                float* p = part + (8 * mb + 2 * j) * TILE_N;
+                facc[mb][0] += p[row_lo]; facc[mb][1] += p[TILE_N + row_lo];
+                facc[mb][2] += p[row_hi]; facc[mb][3] += p[TILE_N + row_hi];
+                if (S > 1) {
+                    p[row_lo] = facc[mb][0]; p[TILE_N + row_lo] = facc[mb][1];
+                    p[row_hi] = facc[mb][2]; p[TILE_N + row_hi] = facc[mb][3];
+                }
             }
         }
     }
@@ -261,39 +272,42 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
         }
         return;
     }
-    if (warp < CL_ROW_WARPS) {
-        // push this slice's partials to the CTAs that own them: slot `slice` of the owner's buffer
-        const int T = M * TILE_N, chunk = (T + S - 1) / S;
+    // The tile's M x 128 sums, as M*32 pieces of four channels, are split into S contiguous shares.
+    const int T4 = M * (TILE_N / 4), chunk4 = (T4 + S - 1) / S;
+    const int lo4 = slice * chunk4;
+    const int cnt4 = (T4 - lo4) < chunk4 ? (T4 - lo4) : chunk4;       // may be <= 0 for the last ranks
+    // the token scale of this thread's first output piece: loaded now, needed after the barrier
+    float t_first = 0.0f;
+    if (tid < cnt4) t_first = __half2float(__ushort_as_half(__ldcg(sa + ((lo4 + tid) >> 5))));
+    __syncthreads();           // the CTA's partial sums are complete in shared memory
+    {
+        // push every piece to the CTA that owns it: slot `slice` of the owner's buffer
+        const float4* part4 = reinterpret_cast<const float4*>(smem + L.set_off);
         const uint32_t red_addr = smem_base + L.red_off;
-        auto push = [&](int m, int nrow, float v) {
-            if (m < M) {
-                const int idx = m * TILE_N + nrow, owner = idx / chunk;
-                const uint32_t off = (uint32_t)(slice * chunk + idx - owner * chunk) * 4u;
-                ptx::st_dsmem_f32(ptx::map_to_cta(red_addr + off, (uint32_t)owner), v);
-            }
-        };
-#pragma unroll
-        for (int mb = 0; mb < MB; ++mb) {
-            const int m0 = 8 * mb + 2 * j;
-            push(m0, row_lo, facc[mb][0]);
-            push(m0 + 1, row_lo, facc[mb][1]);
-            push(m0, row_hi, facc[mb][2]);
-            push(m0 + 1, row_hi, facc[mb][3]);
+        for (int q = tid; q < T4; q += CL_THREADS) {
+            const int owner = q / chunk4;
+            const uint32_t off = (uint32_t)(slice * chunk4 + q - owner * chunk4) * 16u;
+            ptx::st_dsmem_f32x4(ptx::map_to_cta(red_addr + off, (uint32_t)owner), part4[q]);
         }
     }
     __syncwarp();
     ptx::cluster_sync();       // arrive.release after the pushes, wait.acquire before the sums
     {
-        const int T = M * TILE_N, chunk = (T + S - 1) / S;
-        const int lo = slice * chunk;
-        const int cnt = (T - lo) < chunk ? (T - lo) : chunk;          // may be <= 0 for the last ranks
-        const float* red = reinterpret_cast<const float*>(smem + L.red_off);
-        for (int i = tid; i < cnt; i += CL_THREADS) {
-            float acc = 0.0f;
-            for (int s = 0; s < S; ++s) acc += red[s * chunk + i];    // rank order: deterministic
-            const int idx = lo + i, m = idx / TILE_N, nn = idx % TILE_N;
-            const float t = __half2float(__ushort_as_half(__ldcg(sa + m)));
-            y[(size_t)m * N + (size_t)ntile * TILE_N + nn] = __float2bfloat16_rn(acc * t);
+        const float4* red4 = reinterpret_cast<const float4*>(smem + L.red_off);
+        for (int i = tid; i < cnt4; i += CL_THREADS) {
+            float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            for (int s = 0; s < S; ++s) {                              // rank order: deterministic
+                const float4 v = red4[s * chunk4 + i];
+                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            }
+            const int m = (lo4 + i) >> 5, nn = ((lo4 + i) & 31) * 4;
+            const float t = (i == tid) ? t_first : __half2float(__ushort_as_half(__ldcg(sa + m)));
+            __nv_bfloat162 o01 = __floats2bfloat162_rn(acc.x * t, acc.y * t);
+            __nv_bfloat162 o23 = __floats2bfloat162_rn(acc.z * t, acc.w * t);
+            uint2 o;
+            o.x = *reinterpret_cast<uint32_t*>(&o01);
+            o.y = *reinterpret_cast<uint32_t*>(&o23);
+            *reinterpret_cast<uint2*>(y + (size_t)m * N + (size_t)ntile * TILE_N + nn) = o;
         }
     }
 }
