@@ -9,10 +9,11 @@
 //  * a producer warp issues the copies; the weight copies of the first R stages are issued before
 //    griddepcontrol.wait, so under programmatic dependent launch the weight stream of this
 //    kernel overlaps the tail of the previous kernel in the stream.
-//  * sixteen consumer warps in two sets of eight (even / odd groups of the slice; a set's warp owns
-//    16 of the 128 rows): mma.sync m16n8k32 (u8 x s8 -> s32), weights as the 16-row operand;
-//    D = P - z * sum(q_a) with the group sums from the quantise kernel; fp32 group scales; the odd
-//    set's partial sums are added to the even set's through shared memory (fixed order).
+//  * sixteen consumer warps in two sets of eight or four sets of four (set s takes groups s,
+//    s + sets, ... of the slice; a set's warp owns one or two blocks of 16 of the 128 rows):
+//    mma.sync m16n8k32 (u8 x s8 -> s32), weights as the 16-row operand; D = P - z * sum(q_a) with
+//    the group sums from the quantise kernel; fp32 group scales; the sets' partial sums are added
+//    through shared memory (fixed order).
 //  * reduction: the tile's M x 128 outputs are split into S contiguous shares, one per CTA of the
 //    cluster.  A CTA lays its fp32 partials out as [token][channel] in its own shared memory and
 //    pushes them in 16-byte pieces into the owners' shared memory (slot = pusher's rank) with
@@ -34,7 +35,7 @@ namespace w4a8 {
 namespace {
 
 constexpr int CL_ROW_WARPS = 8;                           // 16 weight rows each: one 128-row blob
-constexpr int CL_CONSUMER_WARPS = 2 * CL_ROW_WARPS;        // two sets: even and odd groups of the slice
+constexpr int CL_CONSUMER_WARPS = 2 * CL_ROW_WARPS;        // split into warp sets that take groups in turn
 constexpr int CL_THREADS = (CL_CONSUMER_WARPS + 1) * 32;   // + one producer warp
 constexpr int CL_MAX_STAGES = 12;
 constexpr int CL_BLOB_STRIDE = 8704;                       // BLOB_BYTES rounded up to a multiple of 128
@@ -43,7 +44,10 @@ constexpr int CL_MAX_S = 8;
 struct ClLayout {
     int act_off, blob_off, bar_off, asum_off, red_off, set_off, misc_off, total;
 };
-__host__ __device__ inline ClLayout cl_layout(int mb, int stages, int ng_max) {
+// warp sets of a kernel whose warps own rb blocks of 16 rows each, and the buffers of partial sums
+__host__ __device__ constexpr int cl_sets(int rb) { return 2 * rb; }
+__host__ __device__ constexpr int cl_parts(int mb, int rb) { return (mb <= 2 && mb * cl_sets(rb) <= 8) ? cl_sets(rb) : 1; }
+__host__ __device__ inline ClLayout cl_layout(int mb, int rb, int stages, int ng_max) {
     ClLayout L;
     L.act_off = 0;                                            // stages x (8*mb rows x 128 B), 1024-aligned
     L.blob_off = L.act_off + stages * 1024 * mb;
@@ -51,7 +55,7 @@ __host__ __device__ inline ClLayout cl_layout(int mb, int stages, int ng_max) {
     L.asum_off = L.bar_off + 2 * CL_MAX_STAGES * 8;
     L.red_off = (L.asum_off + 8 * mb * ng_max * 4 + 15) & ~15;
     L.set_off = L.red_off + (8 * mb * (TILE_N / 4) + CL_MAX_S) * 16;   // S slots x ceil(M*32/S) float4
-    L.misc_off = L.set_off + 8 * mb * TILE_N * 4;                 // this CTA's partial sums, [token][channel] fp32
+    L.misc_off = L.set_off + cl_parts(mb, rb) * 8 * mb * TILE_N * 4;   // partial sums, [token][channel] fp32
     L.total = L.misc_off + 16;
     return L;
 }
@@ -67,7 +71,7 @@ __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, 
 // MINB = 2 caps the registers so that two CTAs fit on an SM: wanted when a launch has more CTAs than
 // SMs anyway (they then share SMs instead of queueing); with fewer CTAs than SMs it only invites the
 // cluster scheduler to pack two of them onto one SM and leave others idle.
-template <int MB, int MINB>
+template <int MB, int MINB, int RB>
 __global__ void __launch_bounds__(CL_THREADS, MINB)
 gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t* __restrict__ sa,
                     const int32_t* __restrict__ asum, const uint8_t* __restrict__ packed,
@@ -78,9 +82,13 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-    const ClLayout L = cl_layout(MB, stages, ng_max);
+    const ClLayout L = cl_layout(MB, RB, stages, ng_max);
     constexpr int MP = 8 * MB;
     constexpr uint32_t ACT_BYTES = MP * GROUP;
+    constexpr int NSETS = cl_sets(RB);                    // warp sets: set s takes groups s, s + NSETS, ...
+    constexpr int WPS = CL_CONSUMER_WARPS / NSETS;        // warps per set, RB blocks of 16 rows each
+    constexpr int NPARTS = cl_parts(MB, RB);              // buffers of partial sums: one per set, or one
+    static_assert(NPARTS == NSETS || RB == 1, "in-place merge is written for two sets");
 
     const int G = K / GROUP;
     const int ntile = blockIdx.x / S;
@@ -99,7 +107,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
         *abort_flag = 0;
         for (int s = 0; s < stages; ++s) {
             ptx::mbar_init(full_bar(s), 1);
-            ptx::mbar_init(empty_bar(s), CL_ROW_WARPS);              // the one set that consumed the stage
+            ptx::mbar_init(empty_bar(s), WPS);                       // the one set that consumed the stage
         }
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tmap_qa);
@@ -117,12 +125,14 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
     // older grid that shared this SM could otherwise be stale.
     ptx::pdl_wait();
 
-    float facc[MB][4];
+    float facc[RB][MB][4];
 #pragma unroll
-    for (int mb = 0; mb < MB; ++mb) facc[mb][0] = facc[mb][1] = facc[mb][2] = facc[mb][3] = 0.0f;
+    for (int b = 0; b < RB; ++b)
+#pragma unroll
+        for (int mb = 0; mb < MB; ++mb) facc[b][mb][0] = facc[b][mb][1] = facc[b][mb][2] = facc[b][mb][3] = 0.0f;
     const int r = lane >> 2, j = lane & 3;
-    const int row_lo = (warp & 7) * 16 + r, row_hi = row_lo + 8;
-    const int set = (warp >> 3) & 1;
+    const int set = (warp / WPS) % NSETS;
+    const int row0 = (warp % WPS) * (16 * RB) + r;        // block b of this warp: rows row0 + 16b and + 8
 
     if (warp == CL_CONSUMER_WARPS) {
         // ------------------------------------------------------------------ producer ----
@@ -154,63 +164,67 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
         bool ok = true;
         int s = set;
         uint32_t phase = 0;
-        for (int gi = set; gi < ng; gi += 2, s += 2) {
+        for (int gi = set; gi < ng; gi += NSETS, s += NSETS) {
             while (s >= stages) { s -= stages; phase ^= 1; }
             ok = ptx::mbar_wait(full_bar(s), phase, abort_flag);
             if (!ok) break;
             const uint8_t* blob = smem + L.blob_off + s * CL_BLOB_STRIDE;
             const uint8_t* act = smem + L.act_off + s * 1024 * MB;
-            const uint4 wa = *reinterpret_cast<const uint4*>(blob + row_lo * 64 + j * 16);
-            const uint4 wb = *reinterpret_cast<const uint4*>(blob + row_hi * 64 + j * 16);
-            const uint32_t wlo[4] = {wa.x, wa.y, wa.z, wa.w}, whi[4] = {wb.x, wb.y, wb.z, wb.w};
-            uint32_t a[4][4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                a[q][0] = wlo[q] & 0x0F0F0F0Fu;            // row_lo, k = 32j + 8q + 0..3
-                a[q][1] = whi[q] & 0x0F0F0F0Fu;            // row_hi, same k
-                a[q][2] = (wlo[q] >> 4) & 0x0F0F0F0Fu;     // row_lo, k = 32j + 8q + 4..7
-                a[q][3] = (whi[q] >> 4) & 0x0F0F0F0Fu;     // row_hi
-            }
-            const uint16_t* sc = reinterpret_cast<const uint16_t*>(blob + BLOB_SCALE_OFF);
-            const float s_lo = __half2float(__ushort_as_half(sc[row_lo]));
-            const float s_hi = __half2float(__ushort_as_half(sc[row_hi]));
-            const int z_lo = (blob[BLOB_ZERO_OFF + (row_lo >> 1)] >> ((row_lo & 1) * 4)) & 0xF;
-            const int z_hi = (blob[BLOB_ZERO_OFF + (row_hi >> 1)] >> ((row_hi & 1) * 4)) & 0xF;
-#pragma unroll
-            for (int mb = 0; mb < MB; ++mb) {
-                // token row 8*mb + r of the stage: 128 B, 16-byte chunks XOR-swizzled by the row index
-                const uint8_t* arow = act + mb * 1024 + r * 128;
-                const uint4 b0 = *reinterpret_cast<const uint4*>(arow + (((2 * j) ^ r) << 4));
-                const uint4 b1 = *reinterpret_cast<const uint4*>(arow + (((2 * j + 1) ^ r) << 4));
-                const uint32_t bq[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-                // four independent MMAs (one per k-step) instead of a dependent chain of four
-                int cq[4][4];
+            for (int b = 0; b < RB; ++b) {
+                const int row_lo = row0 + 16 * b, row_hi = row_lo + 8;
+                const uint4 wa = *reinterpret_cast<const uint4*>(blob + row_lo * 64 + j * 16);
+                const uint4 wb = *reinterpret_cast<const uint4*>(blob + row_hi * 64 + j * 16);
+                const uint32_t wlo[4] = {wa.x, wa.y, wa.z, wa.w}, whi[4] = {wb.x, wb.y, wb.z, wb.w};
+                uint32_t a[4][4];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    cq[q][0] = cq[q][1] = cq[q][2] = cq[q][3] = 0;
-                    mma_u8s8(cq[q], a[q][0], a[q][1], a[q][2], a[q][3], bq[2 * q], bq[2 * q + 1]);
+                    a[q][0] = wlo[q] & 0x0F0F0F0Fu;            // row_lo, k = 32j + 8q + 0..3
+                    a[q][1] = whi[q] & 0x0F0F0F0Fu;            // row_hi, same k
+                    a[q][2] = (wlo[q] >> 4) & 0x0F0F0F0Fu;     // row_lo, k = 32j + 8q + 4..7
+                    a[q][3] = (whi[q] >> 4) & 0x0F0F0F0Fu;     // row_hi
                 }
-                int c[4];
+                const uint16_t* sc = reinterpret_cast<const uint16_t*>(blob + BLOB_SCALE_OFF);
+                const float s_lo = __half2float(__ushort_as_half(sc[row_lo]));
+                const float s_hi = __half2float(__ushort_as_half(sc[row_hi]));
+                const int z_lo = (blob[BLOB_ZERO_OFF + (row_lo >> 1)] >> ((row_lo & 1) * 4)) & 0xF;
+                const int z_hi = (blob[BLOB_ZERO_OFF + (row_hi >> 1)] >> ((row_hi & 1) * 4)) & 0xF;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) c[e] = (cq[0][e] + cq[1][e]) + (cq[2][e] + cq[3][e]);
-                const int m0 = 8 * mb + 2 * j;
-                const int A0 = asum_s[m0 * ng_max + gi], A1 = asum_s[(m0 + 1) * ng_max + gi];
-                const int d0 = c[0] - z_lo * A0, d1 = c[1] - z_lo * A1;
-                const int d2 = c[2] - z_hi * A0, d3 = c[3] - z_hi * A1;
-                facc[mb][0] = fmaf(s_lo, (float)d0, facc[mb][0]);
-                facc[mb][1] = fmaf(s_lo, (float)d1, facc[mb][1]);
-                facc[mb][2] = fmaf(s_hi, (float)d2, facc[mb][2]);
-                facc[mb][3] = fmaf(s_hi, (float)d3, facc[mb][3]);
-                if (debug_partials) {
-                    const size_t n_lo = (size_t)ntile * TILE_N + row_lo, n_hi = n_lo + 8;
-                    const int g = g0 + gi;
-                    if (m0 < M) {
-                        debug_partials[((size_t)m0 * G + g) * N + n_lo] = d0;
-                        debug_partials[((size_t)m0 * G + g) * N + n_hi] = d2;
+                for (int mb = 0; mb < MB; ++mb) {
+                    // token row 8*mb + r of the stage: 128 B, 16-byte chunks XOR-swizzled by the row index
+                    const uint8_t* arow = act + mb * 1024 + r * 128;
+                    const uint4 b0 = *reinterpret_cast<const uint4*>(arow + (((2 * j) ^ r) << 4));
+                    const uint4 b1 = *reinterpret_cast<const uint4*>(arow + (((2 * j + 1) ^ r) << 4));
+                    const uint32_t bq[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                    // four independent MMAs (one per k-step) instead of a dependent chain of four
+                    int cq[4][4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        cq[q][0] = cq[q][1] = cq[q][2] = cq[q][3] = 0;
+                        mma_u8s8(cq[q], a[q][0], a[q][1], a[q][2], a[q][3], bq[2 * q], bq[2 * q + 1]);
                     }
-                    if (m0 + 1 < M) {
-                        debug_partials[((size_t)(m0 + 1) * G + g) * N + n_lo] = d1;
-                        debug_partials[((size_t)(m0 + 1) * G + g) * N + n_hi] = d3;
+                    int c[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) c[e] = (cq[0][e] + cq[1][e]) + (cq[2][e] + cq[3][e]);
+                    const int m0 = 8 * mb + 2 * j;
+                    const int A0 = asum_s[m0 * ng_max + gi], A1 = asum_s[(m0 + 1) * ng_max + gi];
+                    const int d0 = c[0] - z_lo * A0, d1 = c[1] - z_lo * A1;
+                    const int d2 = c[2] - z_hi * A0, d3 = c[3] - z_hi * A1;
+                    facc[b][mb][0] = fmaf(s_lo, (float)d0, facc[b][mb][0]);
+                    facc[b][mb][1] = fmaf(s_lo, (float)d1, facc[b][mb][1]);
+                    facc[b][mb][2] = fmaf(s_hi, (float)d2, facc[b][mb][2]);
+                    facc[b][mb][3] = fmaf(s_hi, (float)d3, facc[b][mb][3]);
+                    if (debug_partials) {
+                        const size_t n_lo = (size_t)ntile * TILE_N + row_lo, n_hi = n_lo + 8;
+                        const int g = g0 + gi;
+                        if (m0 < M) {
+                            debug_partials[((size_t)m0 * G + g) * N + n_lo] = d0;
+                            debug_partials[((size_t)m0 * G + g) * N + n_hi] = d2;
+                        }
+                        if (m0 + 1 < M) {
+                            debug_partials[((size_t)(m0 + 1) * G + g) * N + n_lo] = d1;
+                            debug_partials[((size_t)(m0 + 1) * G + g) * N + n_hi] = d3;
+                        }
                     }
                 }
             }
@@ -222,28 +236,37 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
             for (int st = 0; st < stages; ++st)
                 for (int spin = 0; spin < (1 << 16) && !ptx::mbar_try_wait(full_bar(st), 0); ++spin) {}
         }
-        // odd-group partials join the even-group ones (even + odd: fixed order) in a [token][channel]
-        // buffer, from which the exchange below pushes 16-byte pieces
+        // The CTA's partial sums go to shared memory as [token][channel]: the exchange below moves
+        // 16-byte pieces of that layout.  With few tokens each warp set has a buffer of its own and
+        // the two are added (even + odd: fixed order) when a piece is read; otherwise the odd set
+        // writes, the even set adds its own values in place.
         float* part = reinterpret_cast<float*>(smem + L.set_off);
-        if (set == 1) {
+        auto put = [&](float* buf) {
 #pragma unroll
-            for (int mb = 0; mb < MB; ++mb) {
-                float* p = part + (8 * mb + 2 * j) * TILE_N;
-                p[row_lo] = facc[mb][0]; p[TILE_N + row_lo] = facc[mb][1];
-                p[row_hi] = facc[mb][2]; p[TILE_N + row_hi] = facc[mb][3];
-            }
-        }
-        ptx::named_bar_sync(1, CL_CONSUMER_WARPS * 32);
-        if (set == 0) {
+            for (int b = 0; b < RB; ++b) {
+                const int row_lo = row0 + 16 * b, row_hi = row_lo + 8;
 #pragma unroll
-            for (int mb = 0; mb < MB; ++mb) {
-                float* p = part + (8 * mb + 2 * j) * TILE_N;
-                facc[mb][0] += p[row_lo]; facc[mb][1] += p[TILE_N + row_lo];
-                facc[mb][2] += p[row_hi]; facc[mb][3] += p[TILE_N + row_hi];
-                if (S > 1) {
-                    p[row_lo] = facc[mb][0]; p[TILE_N + row_lo] = facc[mb][1];
-                    p[row_hi] = facc[mb][2]; p[TILE_N + row_hi] = facc[mb][3];
+                for (int mb = 0; mb < MB; ++mb) {
+                    float* p = buf + (8 * mb + 2 * j) * TILE_N;
+                    p[row_lo] = facc[b][mb][0]; p[TILE_N + row_lo] = facc[b][mb][1];
+                    p[row_hi] = facc[b][mb][2]; p[TILE_N + row_hi] = facc[b][mb][3];
                 }
+            }
+        };
+        if (NPARTS > 1) {
+            put(part + set * (MP * TILE_N));
+        } else {
+            if (set == 1) put(part);
+            ptx::named_bar_sync(1, CL_CONSUMER_WARPS * 32);
+            if (set == 0) {
+                const int row_lo = row0, row_hi = row_lo + 8;
+#pragma unroll
+                for (int mb = 0; mb < MB; ++mb) {
+                    const float* p = part + (8 * mb + 2 * j) * TILE_N;
+                    facc[0][mb][0] += p[row_lo]; facc[0][mb][1] += p[TILE_N + row_lo];
+                    facc[0][mb][2] += p[row_hi]; facc[0][mb][3] += p[TILE_N + row_hi];
+                }
+                put(part);
             }
         }
     }
@@ -251,27 +274,6 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
 
     __syncwarp();
     ptx::cluster_wait();       // every CTA of the cluster has started: its shared memory may be written
-    if (S == 1) {
-        // a single slice owns the whole K range: its partials are the result, no exchange needed
-        if (warp < CL_ROW_WARPS) {
-            __nv_bfloat16* ycol = y + (size_t)ntile * TILE_N;
-#pragma unroll
-            for (int mb = 0; mb < MB; ++mb) {
-                const int m0 = 8 * mb + 2 * j;
-                if (m0 < M) {
-                    const float t = __half2float(__ushort_as_half(__ldcg(sa + m0)));
-                    ycol[(size_t)m0 * N + row_lo] = __float2bfloat16_rn(facc[mb][0] * t);
-                    ycol[(size_t)m0 * N + row_hi] = __float2bfloat16_rn(facc[mb][2] * t);
-                }
-                if (m0 + 1 < M) {
-                    const float t = __half2float(__ushort_as_half(__ldcg(sa + m0 + 1)));
-                    ycol[(size_t)(m0 + 1) * N + row_lo] = __float2bfloat16_rn(facc[mb][1] * t);
-                    ycol[(size_t)(m0 + 1) * N + row_hi] = __float2bfloat16_rn(facc[mb][3] * t);
-                }
-            }
-        }
-        return;
-    }
     // The tile's M x 128 sums, as M*32 pieces of four channels, are split into S contiguous shares.
     const int T4 = M * (TILE_N / 4), chunk4 = (T4 + S - 1) / S;
     const int lo4 = slice * chunk4;
@@ -280,25 +282,39 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
     float t_first = 0.0f;
     if (tid < cnt4) t_first = __half2float(__ushort_as_half(__ldcg(sa + ((lo4 + tid) >> 5))));
     __syncthreads();           // the CTA's partial sums are complete in shared memory
-    {
+    const float4* part4 = reinterpret_cast<const float4*>(smem + L.set_off);
+    auto piece = [&](int q) {
+        float4 v = part4[q];
+#pragma unroll
+        for (int p = 1; p < NPARTS; ++p) {                 // set order: deterministic
+            const float4 o = part4[q + p * MP * (TILE_N / 4)];
+            v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+        }
+        return v;
+    };
+    if (S > 1) {
         // push every piece to the CTA that owns it: slot `slice` of the owner's buffer
-        const float4* part4 = reinterpret_cast<const float4*>(smem + L.set_off);
         const uint32_t red_addr = smem_base + L.red_off;
         for (int q = tid; q < T4; q += CL_THREADS) {
             const int owner = q / chunk4;
             const uint32_t off = (uint32_t)(slice * chunk4 + q - owner * chunk4) * 16u;
-            ptx::st_dsmem_f32x4(ptx::map_to_cta(red_addr + off, (uint32_t)owner), part4[q]);
+            ptx::st_dsmem_f32x4(ptx::map_to_cta(red_addr + off, (uint32_t)owner), piece(q));
         }
+        __syncwarp();
+        ptx::cluster_sync();   // arrive.release after the pushes, wait.acquire before the sums
     }
-    __syncwarp();
-    ptx::cluster_sync();       // arrive.release after the pushes, wait.acquire before the sums
     {
         const float4* red4 = reinterpret_cast<const float4*>(smem + L.red_off);
         for (int i = tid; i < cnt4; i += CL_THREADS) {
-            float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            for (int s = 0; s < S; ++s) {                              // rank order: deterministic
-                const float4 v = red4[s * chunk4 + i];
-                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            float4 acc;
+            if (S == 1) {
+                acc = piece(i);            // a single slice owns the whole K range: no exchange
+            } else {
+                acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                for (int s = 0; s < S; ++s) {                          // rank order: deterministic
+                    const float4 v = red4[s * chunk4 + i];
+                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                }
             }
             const int m = (lo4 + i) >> 5, nn = ((lo4 + i) & 31) * 4;
             const float t = (i == tid) ? t_first : __half2float(__ushort_as_half(__ldcg(sa + m)));
@@ -312,7 +328,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
     }
 }
 
-template <int MB, int MINB>
+template <int MB, int MINB, int RB>
 cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed, void* y,
                       int M, int N, int K, int S, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
     const int G = K / GROUP;
@@ -323,19 +339,20 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
     const int waves = (ctas + sms - 1) / sms;
     int budget = waves <= 1 ? 110 * 1024 : (220 * 1024) / waves;
     if (budget < 40 * 1024) budget = 40 * 1024;
-    const int fixed = cl_layout(MB, 0, ng_max).total + 1024;
+    const int fixed = cl_layout(MB, RB, 0, ng_max).total + 1024;
     int stages = (budget - fixed) / (CL_BLOB_STRIDE + 1024 * MB);
     if (stages > CL_MAX_STAGES) stages = CL_MAX_STAGES;
     if (stages >= ng_max) {
         stages = ng_max;                       // every stage is used once
     } else {
-        // Stages are reused.  Even and odd groups go to different warp sets and a parity wait can
+        // Stages are reused.  Consecutive groups go to different warp sets and a parity wait can
         // only tell consecutive uses of a barrier apart, so each stage must always serve the same
-        // set: the ring length has to be even.
-        stages &= ~1;
-        if (stages < 2) stages = 2;
+        // set: the ring length has to be a multiple of the number of sets.
+        constexpr int NSETS = cl_sets(RB);
+        stages -= stages % NSETS;
+        if (stages < NSETS) stages = NSETS;
     }
-    const ClLayout L = cl_layout(MB, stages, ng_max);
+    const ClLayout L = cl_layout(MB, RB, stages, ng_max);
     const size_t smem = (size_t)L.total + 1024;
     if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
     int dev = 0;
@@ -344,7 +361,7 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     static bool attr_done[64] = {false};
     if (!attr_done[dev]) {
-        e = cudaFuncSetAttribute(gemm_cluster_kernel<MB, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        e = cudaFuncSetAttribute(gemm_cluster_kernel<MB, MINB, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         attr_done[dev] = true;
     }
@@ -369,7 +386,7 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
     cfg.attrs = attrs;
     cfg.numAttrs = 3;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    return cudaLaunchKernelEx(&cfg, gemm_cluster_kernel<MB, MINB>, tmap, sa, asum, static_cast<const uint8_t*>(packed),
+    return cudaLaunchKernelEx(&cfg, gemm_cluster_kernel<MB, MINB, RB>, tmap, sa, asum, static_cast<const uint8_t*>(packed),
                               static_cast<__nv_bfloat16*>(y), M, N, K, S, ng_max, stages,
                               reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF), debug_partials);
 }
@@ -387,12 +404,11 @@ int cluster_num_slices(int M, int N, int K) {
         if (v >= 1 && v <= CL_MAX_S && v <= G) return v;
     }
     int s;
-    if (M <= 8) {
-        s = ((sms * 14) / 10 + tiles / 2) / tiles;
-    } else {
-        s = 1;
-        while (2 * s <= CL_MAX_S && tiles * 2 * s <= (sms * 9) / 10) s *= 2;
-    }
+    // Powers of two only (clusters of other sizes schedule worse).  Up to 8 tokens two CTAs share an
+    // SM, so up to 1.75 CTAs per SM still run as one wave; above that one CTA per SM.
+    const int cta_limit = M <= 8 ? (sms * 7) / 4 : (sms * 9) / 10;
+    s = 1;
+    while (2 * s <= CL_MAX_S && tiles * 2 * s <= cta_limit) s *= 2;
     if (s > CL_MAX_S) s = CL_MAX_S;
     if (s > G) s = G;
     if (s < 1) s = 1;
@@ -403,14 +419,21 @@ cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int3
                                 void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream) {
     const int S = cluster_num_slices(M, N, K);
-    if (M <= 8) return launch_mb<1, 2>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);   // two launches co-resident
+    if (M <= 8) {
+        // two launches co-resident.  Four warp sets (each warp two blocks of 16 rows) when a slice is
+        // long enough to give every set at least two groups: more groups in flight per CTA and the
+        // activation fragments are loaded once for both blocks.
+        const int ng_max = (K / GROUP + S - 1) / S;
+        if (ng_max >= 8) return launch_mb<1, 2, 2>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+        return launch_mb<1, 2, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+    }
     if (M <= 16) {
         if ((N / TILE_N) * S > device_sm_count())
-            return launch_mb<2, 2>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
-        return launch_mb<2, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+            return launch_mb<2, 2, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+        return launch_mb<2, 1, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
     }
-    if (M <= 32) return launch_mb<4, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
-    return launch_mb<8, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+    if (M <= 32) return launch_mb<4, 1, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+    return launch_mb<8, 1, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
 }
 
 }  // namespace w4a8
