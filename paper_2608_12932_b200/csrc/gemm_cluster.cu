@@ -196,20 +196,30 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
                     const uint4 b0 = *reinterpret_cast<const uint4*>(arow + (((2 * j) ^ r) << 4));
                     const uint4 b1 = *reinterpret_cast<const uint4*>(arow + (((2 * j + 1) ^ r) << 4));
                     const uint32_t bq[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-                    // four independent MMAs (one per k-step) instead of a dependent chain of four
-                    int cq[4][4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        cq[q][0] = cq[q][1] = cq[q][2] = cq[q][3] = 0;
-                        mma_u8s8(cq[q], a[q][0], a[q][1], a[q][2], a[q][3], bq[2 * q], bq[2 * q + 1]);
-                    }
-                    int c[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) c[e] = (cq[0][e] + cq[1][e]) + (cq[2][e] + cq[3][e]);
                     const int m0 = 8 * mb + 2 * j;
                     const int A0 = asum_s[m0 * ng_max + gi], A1 = asum_s[(m0 + 1) * ng_max + gi];
-                    const int d0 = c[0] - z_lo * A0, d1 = c[1] - z_lo * A1;
-                    const int d2 = c[2] - z_hi * A0, d3 = c[3] - z_hi * A1;
+                    int d0, d1, d2, d3;       // D = P - z * sum(q_a)
+                    if (MB == 2) {
+                        // two token blocks give two independent chains: the four MMAs of a block add
+                        // onto one accumulator that starts at the zero-point term (fewer instructions)
+                        int c[4] = {-z_lo * A0, -z_lo * A1, -z_hi * A0, -z_hi * A1};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) mma_u8s8(c, a[q][0], a[q][1], a[q][2], a[q][3], bq[2 * q], bq[2 * q + 1]);
+                        d0 = c[0]; d1 = c[1]; d2 = c[2]; d3 = c[3];
+                    } else {
+                        // four independent MMAs (one per k-step) instead of a dependent chain of four
+                        int cq[4][4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            cq[q][0] = cq[q][1] = cq[q][2] = cq[q][3] = 0;
+                            mma_u8s8(cq[q], a[q][0], a[q][1], a[q][2], a[q][3], bq[2 * q], bq[2 * q + 1]);
+                        }
+                        int c[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) c[e] = (cq[0][e] + cq[1][e]) + (cq[2][e] + cq[3][e]);
+                        d0 = c[0] - z_lo * A0; d1 = c[1] - z_lo * A1;
+                        d2 = c[2] - z_hi * A0; d3 = c[3] - z_hi * A1;
+                    }
                     facc[b][mb][0] = fmaf(s_lo, (float)d0, facc[b][mb][0]);
                     facc[b][mb][1] = fmaf(s_lo, (float)d1, facc[b][mb][1]);
                     facc[b][mb][2] = fmaf(s_hi, (float)d2, facc[b][mb][2]);
