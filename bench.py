@@ -337,7 +337,7 @@ def run_gpu(args):
     _, gt = timer.graph_ms(gemm_only, replays=5, warm=2)
     gemm_us = float(np.median(gt)) * 1e3 / args.steps
     gbytes = wl.algorithmic_bytes_gemm(M, N, K)
-    roof_kernel, roof_us, roof_bytes = "gemm_cluster_kernel<1>", gemm_us, gbytes
+    roof_kernel, roof_us, roof_bytes = "gemm_cluster_kernel<1,2,2>", gemm_us, gbytes
     achieved = roof_bytes / roof_us / 1e3
 
     def quant_only():
@@ -447,7 +447,7 @@ def run_shape(args):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one split-K GEMM launch at the headline shape,
 # from the ncu capture summarised in profiles/gemm_cluster_qkv_M8.md
-TRAFFIC_BYTES_PER_LAUNCH = 13132288
+TRAFFIC_BYTES_PER_LAUNCH = 13144064
 
 
 def main():
