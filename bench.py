@@ -17,7 +17,8 @@ Printed on one JSON line: the step throughput (`value`), the same measured end t
 pinned host buffers through w4a8_linear_host (`e2e`), the roofline of the dominant kernel
 (`roofline`), the CPU oracle timed on this host's cores (`cpu_baseline`), the SM clocks seen
 during the timed region (`clocks`), and - unless --no-sweep - TOPS / GB/s / roofline fraction
-for all four linears of the decoder layer at M = 1...4096 (`sweep`).
+for all four linears of the decoder layer at M = 1...4096 (`sweep`) and the four linears of one layer
+chained in one graph (`layer_chain`).
 
 Multi-GPU: the path does not shard (one GPU per model replica); with --gpus N every rank
 runs the same replica on its own GPU and the value is the sum over ranks (weak scaling).
@@ -243,6 +244,54 @@ def run_sweep(torch, B, peaks, l2_bytes, timer):
     return out
 
 
+def run_layer_chain(torch, B, peaks, l2_bytes, timer):
+    """The four linears of one decoder layer back to back (QKV, O, gate+up, down), each as the public
+    w4a8_linear call (quantise + GEMM) on its own input, in one CUDA graph: what a decoder layer spends in
+    this path per step, launch chain included.  Three cold copies of the layer's weights are visited in turn."""
+    out = []
+    int8_peak = 2.0 * peaks["bf16_tflops"]
+    layer_bytes = sum(K * N // 2 + 5 * (K // 128) * N // 2 for K, N in wl.LAYERS.values())
+    ncopies = copies_for(layer_bytes, l2_bytes)
+    rng = np.random.default_rng(7)
+    m_max = 1024
+    layers = []
+    for lname, (K, N) in wl.LAYERS.items():
+        c = wl.random_codes(rng, m_max, N, K)
+        p0 = B.w4a8_pack_weights(torch.from_numpy(c["qw"]).cuda(), to_dev16(torch, c["sw"], torch.float16),
+                                 torch.from_numpy(c["z"]).cuda())
+        layers.append({"K": K, "N": N, "x": to_dev16(torch, c["x"], torch.bfloat16),
+                       "packed": [p0] + [p0.clone() for _ in range(ncopies - 1)],
+                       "ws": B.new_workspace(m_max, N, K)})
+    for M in (8, 1024):
+        for L in layers:
+            K, N = L["K"], L["N"]
+            L["xm"] = L["x"][:M].contiguous()
+            L["scratch"] = (torch.empty((M, K), dtype=torch.int8, device="cuda"),
+                            torch.empty((M,), dtype=torch.float16, device="cuda"),
+                            torch.empty((M, K // 128), dtype=torch.int32, device="cuda"))
+            L["y"] = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        reps = 4 if M <= 64 else 1
+
+        def body():
+            for _ in range(reps):
+                for c in range(ncopies):
+                    for L in layers:
+                        B.w4a8_linear(L["xm"], L["packed"][c], L["N"], L["ws"], 128, out=L["y"], scratch=L["scratch"])
+        _, times = timer.graph_ms(body, replays=5, warm=2)
+        for L in layers:
+            B.w4a8_check_status(L["ws"])
+        us = min(times) * 1e3 / (reps * ncopies)
+        ops = sum(wl.algorithmic_ops(M, L["N"], L["K"]) for L in layers)
+        nbytes = sum(step_bytes(M, L["N"], L["K"]) for L in layers)
+        t_roof = sum(max(wl.algorithmic_ops(M, L["N"], L["K"]) / (int8_peak * 1e12),
+                         step_bytes(M, L["N"], L["K"]) / (peaks["hbm_gbs"] * 1e9)) for L in layers)
+        out.append({"M": M, "us_per_layer": round(us, 2), "kernels_per_layer": 8, "tops": round(ops / us / 1e6, 1),
+                    "gbs": round(nbytes / us / 1e3, 1), "frac_measured": round(t_roof * 1e6 / us, 3)})
+    del layers
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -386,6 +435,7 @@ def run_gpu(args):
     sweep = None
     if not args.no_sweep and world == 1:
         sweep = run_sweep(torch, B, peaks, l2_bytes, timer)
+        layer_chain = run_layer_chain(torch, B, peaks, l2_bytes, timer)
 
     line = {
         "metric": METRIC, "value": round(value, 2), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
@@ -416,6 +466,7 @@ def run_gpu(args):
     }
     if sweep is not None:
         line["sweep"] = sweep
+        line["layer_chain"] = layer_chain
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
