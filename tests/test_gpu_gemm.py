@@ -178,6 +178,33 @@ def test_zero_point_invariant_and_determinism(mid_case, path, M):
     assert np.array_equal(y1, y2)
 
 
+@pytest.mark.parametrize("path,M", [("splitk", 5), ("splitk", 16), ("splitk_ws", 8), ("tcgen05", 40), ("tcgen05", 209)])
+def test_extreme_codes_zero_points_and_symmetric_scheme(path, M):
+    """Every activation code at +-127 (rows of constant magnitude) against groups whose codes and zero
+    points sit at the ends of their ranges (q - z = +-15: the largest partials, |D| = 243840), the
+    symmetric scheme (z = 8 in every group) and random groups: partials bit-exact, output in tolerance."""
+    rng = np.random.default_rng(11)
+    K, N, g = 1024, 256, 128
+    G = K // g
+    qw = rng.integers(0, 16, size=(N, K), dtype=np.uint8)
+    z = rng.integers(0, 16, size=(G, N), dtype=np.uint8)
+    qw[:, 0 * g:1 * g], z[0] = 15, 0                      # q - z = +15 everywhere
+    qw[:, 1 * g:2 * g], z[1] = 0, 15                      # q - z = -15 everywhere
+    z[2], z[3] = 8, 8                                     # symmetric int4, random codes
+    qw[:, 4 * g:5 * g] = np.where(rng.random((N, g)) < 0.5, 0, 15).astype(np.uint8)
+    z[4] = np.where(rng.random(N) < 0.5, 0, 15).astype(np.uint8)       # codes and zero points at both ends
+    sw = (rng.random((G, N)) * 0.01 + 0.001).astype(np.float16).view(np.uint16)
+    mag = rng.choice(np.array([0.25, 1.0, 3.0, 20.0]), size=(M, 1))
+    sign = np.where(rng.random((M, K)) < 0.5, -1.0, 1.0)
+    sign[0], sign[M - 1] = 1.0, -1.0                      # whole rows at +127 and at -127
+    x = wl.f32_to_bf16_bits((mag * sign).astype(np.float32))
+    case = dict(x=x, qw=qw, sw=sw, z=z, group=g, N=N, K=K)
+    layer = DeviceLayer(case, M)
+    y, D, r = check_case(case, layer, M, path)
+    assert set(np.unique(np.abs(r["qa"]))) == {127}
+    assert D[0, 0].max() == 243840 and D[0, 1].min() == -243840 and D[M - 1, 0].min() == -243840
+
+
 def test_both_paths_give_identical_partials(mid_case):
     case, layer = mid_case
     M = 48

@@ -179,6 +179,35 @@ def test_partials_exhaustive_codes_and_zero_points(impl):
                 assert D[m, 0, n] == (a - zp) * int(qa[m, 0]) + (b - zp) * int(qa[m, 1])
 
 
+@pytest.mark.parametrize("impl", IMPLS)
+def test_extreme_codes_closed_form(impl):
+    """Largest partials a group of 128 can hold: codes 15 (or 0) against zero point 0 (or 15) with every
+    activation code at +-127 give D = +-15 * 127 * 128 = +-243840 by hand; with unit scales and
+    s_a = 1 the output is the sum over groups, bf16-rounded.  The symmetric scheme (z = 8 everywhere)
+    with all codes 8 +- 7 gives +-7 * 127 * 128 = +-113792."""
+    K, g = 512, 128
+    x = np.full((2, K), 127.0)
+    x[1] = -127.0                                           # s_a = fp16(127/127) = 1, q_a = +-127
+    xb = bits_bf16(x)
+    #            group 0      group 1       group 2       group 3
+    code = np.array([15, 0, 15, 1], dtype=np.uint8)         # channel 0
+    zero = np.array([0, 15, 8, 8], dtype=np.uint8)
+    qw = np.repeat(code, g)[None, :].copy()                 # N = 1
+    z = zero[:, None].copy()
+    one = np.full((4, 1), 0x3C00, dtype=np.uint16)
+    if impl == "numpy":
+        r = onp.w4a8_linear(xb, qw, one, z, g)
+    else:
+        r = cfast.w4a8_linear(xb, qw, one, z, g, want_partials=True)
+    assert list(r["sa"]) == [0x3C00, 0x3C00]
+    want = np.array([243840, -243840, 113792, -113792])
+    assert np.array_equal(r["D"][0, :, 0], want) and np.array_equal(r["D"][1, :, 0], -want)
+    assert r["ref"][0, 0] == 0.0 and r["ref"][1, 0] == 0.0            # the four groups cancel exactly
+    # without the last group: 243840 - 243840 + 113792 = 113792 exactly
+    r3 = (onp if impl == "numpy" else cfast).w4a8_linear(xb[:, :384], qw[:, :384], one[:3], z[:3], g)
+    assert r3["ref"][0, 0] == 113792.0 and r3["ref"][1, 0] == -113792.0
+
+
 # ---------------------------------------------- reduction to library routines (dgemm) --
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("name,M", [("tiny", 16), ("mid", 24)])
