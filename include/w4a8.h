@@ -135,6 +135,23 @@ typedef struct {
 } w4a8_plan_info;
 w4a8_status w4a8_plan(int M, int N, int K, int group, w4a8_plan_info* out);
 
+/*
+ * Variant for weights whose scale does not change along K (per-channel scales: the paper does not
+ * give its group size, Sec. 3.4; this is the coarsest choice, group 128 the library's default).
+ * Same packed format and the same per-group zero points; the caller guarantees that the scales of
+ * a channel are equal in every group (only those of the first group are read).  The int32 sums of
+ * all groups then add up in one tensor-memory accumulator and a tile is scaled once:
+ *   y[m,n] = bf16( sa[m] * sw[n] * sum_groups D[m,group,n] )
+ * which equals w4a8_gemm's result up to fp32 rounding order.  tcgen05 kernel for every M.
+ *   debug_sums   NULL, or [M,N] int32 that receives sum_groups D (exact)
+ * K <= 2^19.  Other arguments, alignment, workspace and errors as for w4a8_gemm.
+ */
+w4a8_status w4a8_gemm_per_channel(const int8_t* qa, const uint16_t* sa,
+                                  const void* packed_w, void* y_bf16,
+                                  int M, int N, int K, int group,
+                                  void* workspace, size_t workspace_bytes,
+                                  int32_t* debug_sums, void* stream);
+
 /* w4a8_gemm with the kernel family forced (path-consistency tests, benchmarking). */
 w4a8_status w4a8_gemm_path(w4a8_path path,
                            const int8_t* qa, const uint16_t* sa, const int32_t* asum,

@@ -19,7 +19,8 @@ WORKSPACE_HEADER_BYTES = 4096
 
 EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w4a8_workspace_init",
            "w4a8_pack_weights", "w4a8_unpack_weights", "w4a8_quantize_act", "w4a8_gemm", "w4a8_gemm_path",
-           "w4a8_linear", "w4a8_linear_host", "w4a8_gemm_static_scratch", "w4a8_check_status", "w4a8_plan")
+           "w4a8_linear", "w4a8_linear_host", "w4a8_gemm_static_scratch", "w4a8_check_status", "w4a8_plan",
+           "w4a8_gemm_per_channel")
 
 _lib = None
 
@@ -57,6 +58,8 @@ def lib():
         L.w4a8_gemm.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp, vp]
         L.w4a8_gemm_path.restype = ci
         L.w4a8_gemm_path.argtypes = [ci, vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp, vp]
+        L.w4a8_gemm_per_channel.restype = ci
+        L.w4a8_gemm_per_channel.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp, vp]
         L.w4a8_plan.restype = ci
         L.w4a8_plan.argtypes = [ci, ci, ci, ci, vp]
         L.w4a8_linear.restype = ci
@@ -173,6 +176,23 @@ def w4a8_gemm(qa, sa, asum, packed_w, N, workspace, group=GROUP, out=None, debug
         code = lib().w4a8_gemm_path(path, _ptr(qa), _ptr(sa), _ptr(asum), _ptr(packed_w), _ptr(out), M, N, K, group,
                                     _ptr(workspace), workspace.numel(), _ptr(debug_partials), _stream(stream))
     _check(code, "w4a8_gemm")
+    return out
+
+
+def w4a8_gemm_per_channel(qa, sa, packed_w, N, workspace, group=GROUP, out=None, debug_sums=None, stream=None):
+    """w4a8_gemm for a packed layer whose scales are equal in every group of a channel: one drain per tile."""
+    _dev(qa, torch.int8, "qa"), _dev(sa, torch.float16, "sa")
+    _dev(packed_w, torch.uint8, "packed_w"), _dev(workspace, torch.uint8, "workspace")
+    M, K = qa.shape
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=qa.device)
+    else:
+        _dev(out, torch.bfloat16, "out")
+    if debug_sums is not None:
+        _dev(debug_sums, torch.int32, "debug_sums")
+    _check(lib().w4a8_gemm_per_channel(_ptr(qa), _ptr(sa), _ptr(packed_w), _ptr(out), M, N, K, group,
+                                       _ptr(workspace), workspace.numel(), _ptr(debug_sums), _stream(stream)),
+           "w4a8_gemm_per_channel")
     return out
 
 

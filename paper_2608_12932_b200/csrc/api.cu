@@ -166,6 +166,22 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
     return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
 
+w4a8_status w4a8_gemm_per_channel(const int8_t* qa, const uint16_t* sa, const void* packed_w, void* y_bf16,
+                                  int M, int N, int K, int group, void* workspace, size_t workspace_bytes,
+                                  int32_t* debug_sums, void* stream) {
+    if (!shape_ok(N, K, group) || M < 0 || K > (1 << 19)) return W4A8_ERR_SHAPE;    // int32 sums: 15 * 127 * K < 2^31
+    if (M == 0) return W4A8_OK;
+    if (!qa || !sa || !packed_w || !y_bf16 || !workspace) return W4A8_ERR_NULL;
+    if (!aligned(qa, 16) || !aligned(sa, 2) || !aligned(packed_w, 128) || !aligned(y_bf16, 2) ||
+        !aligned(workspace, 256) || (debug_sums && !aligned(debug_sums, 4)))
+        return W4A8_ERR_ALIGN;
+    if (workspace_bytes < w4a8_workspace_bytes(M, N, K, group)) return W4A8_ERR_WORKSPACE;
+    w4a8_status a = arch_check();
+    if (a != W4A8_OK) return a;
+    return launch_gemm_tcgen05_per_channel(qa, sa, packed_w, y_bf16, M, N, K, workspace, debug_sums,
+                                           static_cast<cudaStream_t>(stream)) == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
 w4a8_status w4a8_plan(int M, int N, int K, int group, w4a8_plan_info* out) {
     if (!shape_ok(N, K, group) || M <= 0) return W4A8_ERR_SHAPE;
     const int sms = device_sm_count(), tiles = N / TILE_N;

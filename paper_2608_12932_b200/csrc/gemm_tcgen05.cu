@@ -91,7 +91,7 @@ struct Cfg {
     static constexpr int B_OFF = 0;
     static constexpr int RAW_OFF = B_OFF + SB * B_BYTES;
     static constexpr int BAR_OFF = RAW_OFF + SR * RAW_STRIDE;
-    static constexpr int NUM_BARS = 2 * SR + SB + SA + 2 + DONE_RING + 2;
+    static constexpr int NUM_BARS = 2 * SR + SB + SA + 2 + DONE_RING + 2 + 2;
     static constexpr int MISC_OFF = (BAR_OFF + NUM_BARS * 8 + 15) & ~15;      // 16-byte aligned: staging is read with 16-byte loads
     static constexpr int W = TILE_M / 2;                                      // accumulator columns (tokens) per drain warp
     static constexpr int NCH = (W + 31) / 32;                                 // 32-column chunks per drain warp (the last may be 8 wide)
@@ -115,7 +115,9 @@ __device__ __forceinline__ uint32_t sub_zero4(uint32_t q, uint32_t kz) {
     return (q + kz) ^ 0x80808080u;
 }
 
-template <int TILE_M, bool DEBUG, bool SPLIT>
+// PC ("per channel"): the scales of a channel are the same in every group, so the integer sums of all
+// groups of a tile add up in one accumulator and the tile is drained once (see w4a8_gemm_per_channel).
+template <int TILE_M, bool DEBUG, bool SPLIT, bool PC = false>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* __restrict__ packed,
                     const uint16_t* __restrict__ sa, __nv_bfloat16* __restrict__ y,
@@ -123,6 +125,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                     int M, int N, int K, int m_tiles, int total_tiles, int S) {
     using C = Cfg<TILE_M>;
     static_assert(!SPLIT || C::SB * C::B_BYTES >= TILE_M * TILE_N * 4 + 64, "the split-K exchange buffer lives in the activation ring");
+    static_assert(!(SPLIT && PC), "the per-channel form is not split along K");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
@@ -140,7 +143,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
     // one event frees the step's weight stage (unpack warps wait for step it - SA), its activation
     // stage (producer waits for step it - SB) and publishes its accumulator (drain warps wait for it).
     const int RAW_FULL = 0, RAW_EMPTY = C::SR, B_FULL = 2 * C::SR, A_FULL = B_FULL + C::SB, ACC_EMPTY = A_FULL + C::SA,
-              DONE = ACC_EMPTY + 2, FINAL = DONE + DONE_RING;
+              DONE = ACC_EMPTY + 2, FINAL = DONE + DONE_RING, TILE_DONE = FINAL + 2;
     auto done_bar = [&](uint32_t step) { return bar(DONE + (int)(step % DONE_RING)); };
     auto done_parity = [](uint32_t step) { return (step / DONE_RING) & 1u; };
     volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(smem + C::MISC_OFF);
@@ -158,6 +161,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
             for (int i = 0; i < 2; ++i) ptx::mbar_init(bar(ACC_EMPTY + i), NUM_DRAIN_WARPS);
             for (int i = 0; i < DONE_RING; ++i) ptx::mbar_init(bar(DONE + i), 1);
             for (int i = 0; i < 2; ++i) ptx::mbar_init(bar(FINAL + i), 1);
+            for (int i = 0; i < 2; ++i) ptx::mbar_init(bar(TILE_DONE + i), 2);      // both MMA issuers
             ptx::fence_mbar_init();
         }
         __syncwarp();
@@ -228,24 +232,34 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
             // descriptor of activation stage 0; a stage and a K slice of 32 bytes are plain
             // additions to its (address >> 4) field
             const uint64_t b_desc0 = ptx::smem_desc_k_sw128(smem_base + C::B_OFF);
-            const uint32_t d_tmem = tmem_base + par * TILE_M;
-            uint32_t it = 0;
+            uint32_t it = 0, tcount = 0;
             bool ok = true;
-            for (int tile = unit; tile < total_tiles && ok; tile += num_units) {
+            for (int tile = unit; tile < total_tiles && ok; tile += num_units, ++tcount) {
+                // PC: both threads add into the buffer of the tile, which the drain warps left zeroed
+                // (integer sums commute, so the order of the two threads' MMAs does not matter)
+                const uint32_t buf = PC ? (tcount & 1u) : par;
+                const uint32_t d_tmem = tmem_base + buf * TILE_M;
+                bool mine = false;
                 for (int g = 0; g < G; ++g, ++it) {
                     if ((it & 1u) != par) continue;
                     const uint32_t sb = it % C::SB, pb = (it / C::SB) & 1;
                     const uint32_t sa_ = it % C::SA, pas = (it / C::SA) & 1;
                     // accumulator drained; activations landed; weights unpacked
-                    if (!(ok = ptx::mbar_wait3_hot(bar(ACC_EMPTY + par), (it >> 1) & 1, bar(B_FULL + sb), pb,
+                    if (!(ok = ptx::mbar_wait3_hot(bar(ACC_EMPTY + buf), ((PC ? tcount : it) >> 1) & 1, bar(B_FULL + sb), pb,
                                                    bar(A_FULL + sa_), pas, abort_flag))) break;
                     ptx::tc_fence_after_sync();
                     const uint64_t bd = b_desc0 + (uint64_t)(sb * (C::B_BYTES / 16));
                     const uint32_t a_tmem = tmem_base + C::A_COL0 + sa_ * A_COLS;
 #pragma unroll
-                    for (int kk = 0; kk < GROUP / 32; ++kk)       // the first K slice overwrites the buffer
-                        ptx::mma_i8_ts(d_tmem, a_tmem + 8 * kk, bd + 2 * kk, idesc, kk ? 1u : 0u);
-                    ptx::tc_commit(done_bar(it));                 // stages consumed, accumulator complete
+                    for (int kk = 0; kk < GROUP / 32; ++kk)       // not PC: the first K slice overwrites the buffer
+                        ptx::mma_i8_ts(d_tmem, a_tmem + 8 * kk, bd + 2 * kk, idesc, (PC || kk) ? 1u : 0u);
+                    ptx::tc_commit(done_bar(it));                 // stages consumed (not PC: accumulator complete)
+                    mine = true;
+                }
+                if (PC && ok) {
+                    // the tile is complete when the MMAs of both threads are: a commit tracks only its own thread's
+                    if (mine) ptx::tc_commit(bar(TILE_DONE + buf));
+                    else ptx::mbar_arrive(bar(TILE_DONE + buf));
                 }
             }
             ptx::tc_commit(bar(FINAL + par));
@@ -306,13 +320,25 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
         const int q = warp & 3, h = (warp - WARP_DRAIN0) >> 2;
         const int n_local = q * 32 + lane;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + h * C::W;
+        // PC: this warp's part of an accumulator buffer back to zero (every MMA of a tile adds)
+        auto zero_fill = [&](uint32_t taddr) {
+#pragma unroll
+            for (int c = 0; c < C::W; c += 8) ptx::tmem_st_32x8(taddr + c, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u);
+            ptx::tmem_st_wait();
+        };
+        if (PC) {
+            zero_fill(lane_taddr);
+            zero_fill(lane_taddr + TILE_M);
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+        }
         if (lane == 0) {                                          // both accumulator buffers start out free
             ptx::mbar_arrive(bar(ACC_EMPTY + 0));
             ptx::mbar_arrive(bar(ACC_EMPTY + 1));
         }
-        uint32_t it = 0;
+        uint32_t it = 0, tcount = 0;
         bool ok = true;
-        for (int tile = unit; tile < total_tiles && ok; tile += num_units) {
+        for (int tile = unit; tile < total_tiles && ok; tile += num_units, ++tcount) {
             int ntile, mtile;
             tile_of(tile, ntile, mtile);
             const int n = ntile * TILE_N + n_local;
@@ -328,7 +354,41 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 sa_w[i] = (m_base + i < M) ? __half2float(__ushort_as_half(__ldg(sa + m_base + i))) : 0.0f;
             __syncwarp();
             uint16_t sw_bits = __ldg(reinterpret_cast<const uint16_t*>(sw_ptr));
-            for (int g = 0; g < G; ++g, ++it) {
+            if (PC) {
+                // one drain per tile: the buffer holds the sum of D over all groups (|sum| < 2^31 for K < 2^13 * 128)
+                const uint32_t buf = tcount & 1u;
+                const float sw = __half2float(__ushort_as_half(sw_bits));
+                if (!(ok = ptx::mbar_wait_hot(bar(TILE_DONE + buf), (tcount >> 1) & 1, abort_flag))) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t taddr = lane_taddr + buf * TILE_M;
+                uint32_t v[C::NCH][32];
+#pragma unroll
+                for (int ch = 0; ch < C::NCH; ++ch) {
+                    if (ch == C::NCH - 1 && C::LAST == 8) ptx::tmem_ld_32x8(taddr + ch * 32, reinterpret_cast<uint32_t(&)[8]>(v[ch]));
+                    else ptx::tmem_ld_32x32(taddr + ch * 32, v[ch]);
+                }
+                ptx::tmem_ld_wait();
+                zero_fill(taddr);
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar(ACC_EMPTY + buf));
+#pragma unroll
+                for (int ch = 0; ch < C::NCH; ++ch) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        if (ch * 32 + i < C::W) {
+                            const int32_t di = (int32_t)v[ch][i];
+                            // exact while |sum| < 2^24; beyond that one rounding of relative size 2^-24
+                            facc[ch * 32 + i] = sw * (float)di;
+                            if (DEBUG) {
+                                const int m = m_base + ch * 32 + i;
+                                if (m < M) debug_partials[(size_t)m * N + n] = di;
+                            }
+                        }
+                    }
+                }
+            }
+            for (int g = 0; g < (PC ? 0 : G); ++g, ++it) {
                 const uint32_t buf = it & 1;
                 const float sw = __half2float(__ushort_as_half(sw_bits));
                 if (g + 1 < G) sw_bits = __ldg(reinterpret_cast<const uint16_t*>(sw_ptr + (size_t)(g + 1) * BLOB_BYTES));
@@ -438,7 +498,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
     }
 }
 
-template <int TILE_M, bool DEBUG, bool SPLIT>
+template <int TILE_M, bool DEBUG, bool SPLIT, bool PC = false>
 cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed, void* y, int M, int N, int K, int S,
                         void* workspace, int32_t* debug_partials, cudaStream_t stream) {
     using C = Cfg<TILE_M>;
@@ -453,7 +513,7 @@ cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     const int sms = device_sm_count();
     if (!attr_done[dev]) {
-        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT, PC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  C::SMEM_ALLOC);
         if (e != cudaSuccess) return e;
         attr_done[dev] = true;
@@ -475,7 +535,7 @@ cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT>, tmap, static_cast<const uint8_t*>(packed), sa,
+    return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT, PC>, tmap, static_cast<const uint8_t*>(packed), sa,
                               static_cast<__nv_bfloat16*>(y), debug_partials, reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF),
                               M, N, K, m_tiles, total, S);
 }
@@ -510,17 +570,17 @@ int max_active_clusters(int S) {
     return cached[dev][S] > 0 ? cached[dev][S] : 0;
 }
 
-template <bool DEBUG>
+template <bool DEBUG, bool PC = false>
 cudaError_t launch_plan(int tile_m, int S, const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
                         int M, int N, int K, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
-    if (S > 1) {
+    if (S > 1 && !PC) {
         if (tile_m == 64) return launch_tile<64, DEBUG, true>(qa, sa, packed, y, M, N, K, S, workspace, debug_partials, stream);
         if (tile_m == 128) return launch_tile<128, DEBUG, true>(qa, sa, packed, y, M, N, K, S, workspace, debug_partials, stream);
         return launch_tile<208, DEBUG, true>(qa, sa, packed, y, M, N, K, S, workspace, debug_partials, stream);
     }
-    if (tile_m == 64) return launch_tile<64, DEBUG, false>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
-    if (tile_m == 128) return launch_tile<128, DEBUG, false>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
-    return launch_tile<208, DEBUG, false>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
+    if (tile_m == 64) return launch_tile<64, DEBUG, false, PC>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
+    if (tile_m == 128) return launch_tile<128, DEBUG, false, PC>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
+    return launch_tile<208, DEBUG, false, PC>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
 }
 
 }  // namespace
@@ -531,7 +591,7 @@ cudaError_t launch_plan(int tile_m, int S, const int8_t* qa, const uint16_t* sa,
 // dominates a group, so taller tiles are cheaper per token); a K split into S slices costs
 // TC_SPLIT_NS for the cluster exchange.  Tall tiles win when there are several waves of them, short
 // ones when a tall tiling would leave SMs idle, and a K split when even the shortest tiling does.
-long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split) {
+long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split, int max_split) {
     const int heights[3] = {208, 128, 64};
     const int n_tiles = N / TILE_N, G = K / GROUP;
     long best_ns = -1;
@@ -541,7 +601,7 @@ long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split) {
         if (heights[i] > 64 && M <= heights[i + 1]) continue;        // the next height down already covers M in one tile
         const long tiles = (long)((M + heights[i] - 1) / heights[i]) * n_tiles;
         const long waves = (tiles + sms - 1) / sms;
-        for (int S = 1; S <= TC_MAX_SPLIT; ++S) {
+        for (int S = 1; S <= TC_MAX_SPLIT && S <= max_split; ++S) {
             if (S > 1) {
                 if (tiles * S > sms || G / S < 4) break;
                 const int room = i == 0 ? max_active_clusters<208>(S) : (i == 1 ? max_active_clusters<128>(S) : max_active_clusters<64>(S));
@@ -558,10 +618,22 @@ cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void
                                 int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream) {
     int tile_m = 64, S = 1;
-    tcgen05_plan(M, N, K, device_sm_count(), &tile_m, &S);
+    tcgen05_plan(M, N, K, device_sm_count(), &tile_m, &S, TC_MAX_SPLIT);
     if (debug_partials)
         return launch_plan<true>(tile_m, S, qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
     return launch_plan<false>(tile_m, S, qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+}
+
+// The same pipeline with one drain per tile: for weights whose scale does not change along K.
+// debug_sums, if not null, receives the int32 sum over all groups per (token, channel), [M][N].
+cudaError_t launch_gemm_tcgen05_per_channel(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
+                                            int M, int N, int K, void* workspace, int32_t* debug_sums,
+                                            cudaStream_t stream) {
+    int tile_m = 64, S = 1;
+    tcgen05_plan(M, N, K, device_sm_count(), &tile_m, &S, 1);
+    if (debug_sums)
+        return launch_plan<true, true>(tile_m, 1, qa, sa, packed, y, M, N, K, workspace, debug_sums, stream);
+    return launch_plan<false, true>(tile_m, 1, qa, sa, packed, y, M, N, K, workspace, debug_sums, stream);
 }
 
 }  // namespace w4a8

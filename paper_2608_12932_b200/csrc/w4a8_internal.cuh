@@ -57,7 +57,11 @@ cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int3
 cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
                                 int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream);
-long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split);    // tile height and K split the tcgen05 launcher picks; returns its time estimate (ns)
+cudaError_t launch_gemm_tcgen05_per_channel(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
+                                            int M, int N, int K, void* workspace, int32_t* debug_sums,
+                                            cudaStream_t stream);
+// tile height and K split (at most max_split slices) the tcgen05 launcher picks; returns its time estimate (ns)
+long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split, int max_split = 4);
 bool small_m_prefers_tcgen05(int M, int N, int K, int sms);
 
 }  // namespace w4a8
