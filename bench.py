@@ -203,7 +203,7 @@ def copies_for(nbytes, l2_bytes):
 
 def run_sweep(torch, B, peaks, l2_bytes, timer):
     """All four linears at every M of the sweep: GEMM alone, rotating cold weight copies."""
-    out = []
+    out, out_pc = [], []
     int8_peak = 2.0 * peaks["bf16_tflops"]
     for lname, (K, N) in wl.LAYERS.items():
         case = wl.make_sweep_layer(lname)
@@ -239,9 +239,22 @@ def run_sweep(torch, B, peaks, l2_bytes, timer):
                         "bound": "int8" if t_c_meas > t_m_meas else "hbm",
                         "frac_measured": round(max(t_c_meas, t_m_meas) * 1e6 / us, 3),
                         "frac_nominal": round(max(t_c_nom, t_m_nom) * 1e6 / us, 3)})
+            if M >= 1024:
+                # the same pipeline with one drain per tile (w4a8_gemm_per_channel: scales constant along K;
+                # it reads the first group's scales only, so the timing needs no second set of weights)
+                def body_pc():
+                    for _ in range(reps):
+                        for p in packed:
+                            B.w4a8_gemm_per_channel(qa, sa, p, N, ws, out=y)
+                _, times = timer.graph_ms(body_pc, replays=5, warm=2)
+                B.w4a8_check_status(ws)
+                us = min(times) * 1e3 / (reps * ncopies)
+                out_pc.append({"layer": lname, "M": M, "us": round(us, 2), "tops": round(ops / us / 1e6, 1),
+                               "frac_measured": round(max(t_c_meas, t_m_meas) * 1e6 / us, 3),
+                               "frac_nominal": round(max(t_c_nom, t_m_nom) * 1e6 / us, 3)})
         del packed, packed0, x_all
         torch.cuda.empty_cache()
-    return out
+    return out, out_pc
 
 
 def run_layer_chain(torch, B, peaks, l2_bytes, timer):
@@ -434,7 +447,7 @@ def run_gpu(args):
 
     sweep = None
     if not args.no_sweep and world == 1:
-        sweep = run_sweep(torch, B, peaks, l2_bytes, timer)
+        sweep, sweep_pc = run_sweep(torch, B, peaks, l2_bytes, timer)
         layer_chain = run_layer_chain(torch, B, peaks, l2_bytes, timer)
 
     line = {
@@ -466,6 +479,7 @@ def run_gpu(args):
     }
     if sweep is not None:
         line["sweep"] = sweep
+        line["sweep_per_channel_scales"] = sweep_pc
         line["layer_chain"] = layer_chain
     print(json.dumps(line))
     if world > 1:
