@@ -510,14 +510,17 @@ def run_shape(args):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         qa, sa, asum = B.w4a8_quantize_act(x)
         e0.record()
-        B.w4a8_gemm(qa, sa, asum, packed[i % ncopies], N, ws, out=y)
+        if args.per_channel:
+            B.w4a8_gemm_per_channel(qa, sa, packed[i % ncopies], N, ws, out=y)
+        else:
+            B.w4a8_gemm(qa, sa, asum, packed[i % ncopies], N, ws, out=y)
         e1.record()
         e1.synchronize()
         if i >= args.warmup:
             times.append(e0.elapsed_time(e1) * 1e3)
     B.w4a8_check_status(ws)
     us = float(np.median(times))
-    print(json.dumps({"shape": args.shape, "M": M, "N": N, "K": K, "gemm_us_eager_median": round(us, 2),
+    print(json.dumps({"shape": args.shape, "per_channel_scales": bool(args.per_channel), "M": M, "N": N, "K": K, "gemm_us_eager_median": round(us, 2),
                       "tops": round(wl.algorithmic_ops(M, N, K) / us / 1e6, 1),
                       "gbs": round(wl.algorithmic_bytes_gemm(M, N, K) / us / 1e3, 1), "launches": args.steps}))
 
@@ -536,6 +539,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--shape", default=None, help="LAYER:M, e.g. gate_up:1024 - run only that GEMM (profiling aid)")
+    ap.add_argument("--per-channel", action="store_true", help="with --shape: w4a8_gemm_per_channel instead of w4a8_gemm")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.shape:
