@@ -153,6 +153,21 @@ def test_ring_reuse_many_groups_per_cta():
     check_case(case, layer, 5, "splitk", debug=False)
 
 
+def test_many_token_tiles_and_very_wide_layer():
+    """Index ranges: 97 token tiles of one channel tile (20001 tokens, a ragged last tile), and 296 channel
+    tiles (two per SM on the split-K path, two rounds of tiles on the tensor-core path)."""
+    case = wl.make_layer(256, 128, 39, 20001)
+    layer = DeviceLayer(case, 20001)
+    rng = np.random.default_rng(3)
+    rows = np.unique(np.concatenate([[0, 207, 208, 19967, 19968, 20000], rng.integers(0, 20001, 40)]))
+    check_case(case, layer, 20001, "tcgen05", debug=True, rows=rows)
+    case = wl.make_layer(256, 296 * 128, 40, 300)
+    layer = DeviceLayer(case, 300)
+    check_case(case, layer, 8, "splitk")
+    check_case(case, layer, 16, "splitk")
+    check_case(case, layer, 300, "tcgen05", rows=[0, 1, 207, 208, 299])
+
+
 def test_persistent_tiles_more_than_sms():
     """160 output tiles over at most 148 CTAs: some CTAs run two tiles back to back."""
     case = wl.make_layer(512, 5120, 33, 1024)
