@@ -111,6 +111,10 @@ def test_shape_validation_needs_no_gpu():
     assert L.w4a8_gemm_path(B.PATH_SPLITK_WORKSPACE, None, None, None, None, None, 65, 128, 256, 128, None, 0, None, None) == B.ERR_SHAPE
     assert L.w4a8_gemm_static_scratch(None, None, None, None, None, 65, 128, 256, 128, None) == B.ERR_SHAPE
     assert L.w4a8_gemm_static_scratch(None, None, None, None, None, 8, 128, 256, 128, None) == B.ERR_NULL
+    assert L.w4a8_gemm_per_channel(None, None, None, None, 8, 128, 256, 64, None, 0, None, None) == B.ERR_SHAPE
+    assert L.w4a8_gemm_per_channel(None, None, None, None, 8, 128, (1 << 19) + 128, 128, None, 0, None, None) == B.ERR_SHAPE
+    assert L.w4a8_gemm_per_channel(None, None, None, None, 0, 128, 256, 128, None, 0, None, None) == B.OK
+    assert L.w4a8_gemm_per_channel(None, None, None, None, 8, 128, 256, 128, None, 0, None, None) == B.ERR_NULL
     assert L.w4a8_workspace_init(None, 4096, None) == B.ERR_NULL
     assert L.w4a8_check_status(None, None) == B.ERR_NULL
     # alignment is checked before the device is queried
