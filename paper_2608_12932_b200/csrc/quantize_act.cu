@@ -15,8 +15,7 @@
 namespace w4a8 {
 namespace {
 
-constexpr int QA_THREADS = 256;
-constexpr int QA_CACHE = 6;   // chunks kept in registers per thread: rows up to 12288 read once
+constexpr int QA_CACHE_CHUNKS = 1536;   // 16-byte chunks of a row kept in registers: rows up to 12288 read once
 
 __device__ __forceinline__ uint32_t absmax_bits_bf16x8(const uint4& v, uint32_t run) {
     // bf16 magnitudes order like their 15-bit patterns: keep a packed running max of two lanes
@@ -47,6 +46,9 @@ __device__ __forceinline__ uint2 quant8(const uint4& v, float s, int& sum) {
     return o;
 }
 
+// QA_THREADS threads per token row: 256 for many rows (more rows in flight per SM), 512 or 1024 for fewer
+// (a row's latency chain - load, row maximum, divisions, store - is then shorter per thread).
+template <int QA_THREADS>
 __global__ void __launch_bounds__(QA_THREADS)
 quantize_act_kernel(const uint4* __restrict__ x, int K, uint2* __restrict__ qa,
                     uint16_t* __restrict__ sa, int32_t* __restrict__ asum) {
@@ -60,6 +62,7 @@ quantize_act_kernel(const uint4* __restrict__ x, int K, uint2* __restrict__ qa,
     const uint4* xr = x + (size_t)m * chunks;
     uint2* qr = qa + (size_t)m * chunks;
     const int tid = threadIdx.x;
+    constexpr int QA_CACHE = QA_CACHE_CHUNKS / QA_THREADS;
 
     uint4 cache[QA_CACHE];
     uint32_t run = 0;
@@ -116,14 +119,23 @@ cudaError_t launch_quantize_act(const void* x, int M, int K, int8_t* qa, uint16_
                                 cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)M, 1, 1);
-    cfg.blockDim = dim3(QA_THREADS, 1, 1);
+    // measured on B200 (K = 4096 and 12288): 512 threads per row are best up to 512 rows except between
+    // about 64 and 128 rows, where 1024 are; from 1024 rows on 256 are
+    const int threads = M > 512 ? 256 : ((M > 48 && M <= 192) ? 1024 : 512);
+    cfg.blockDim = dim3((unsigned)threads, 1, 1);
     cfg.stream = stream;
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, quantize_act_kernel, reinterpret_cast<const uint4*>(x), K,
+    if (threads == 1024)
+        return cudaLaunchKernelEx(&cfg, quantize_act_kernel<1024>, reinterpret_cast<const uint4*>(x), K,
+                                  reinterpret_cast<uint2*>(qa), sa, asum);
+    if (threads == 512)
+        return cudaLaunchKernelEx(&cfg, quantize_act_kernel<512>, reinterpret_cast<const uint4*>(x), K,
+                                  reinterpret_cast<uint2*>(qa), sa, asum);
+    return cudaLaunchKernelEx(&cfg, quantize_act_kernel<256>, reinterpret_cast<const uint4*>(x), K,
                               reinterpret_cast<uint2*>(qa), sa, asum);
 }
 

@@ -28,7 +28,9 @@ def assert_quantize_parity(x_bits):
 
 
 @pytest.mark.parametrize("M,K,seed", [(16, 256, 0), (8, 4096, 0), (1, 128, 1), (37, 12288, 2), (5, 16512, 3),
-                                      (1024, 4096, 4), (3, 2048 + 128, 5)])
+                                      (1024, 4096, 4), (3, 2048 + 128, 5),
+                                      # every threads-per-row variant of the kernel, short and long rows
+                                      (100, 4096, 6), (128, 128, 7), (70, 16512, 8), (400, 12288, 9), (513, 1024, 10)])
 def test_quantize_matches_oracle(M, K, seed):
     rng = np.random.default_rng(seed)
     x = rng.standard_normal((M, K), dtype=np.float32)
