@@ -66,7 +66,8 @@ size_t w4a8_packed_bytes(int N, int K, int group);
 
 /*
  * Size in bytes of the scratch workspace w4a8_gemm needs for any M <= M_max on this
- * layer shape (split-K slices, per-tile arrival counters, one status word); 0 for an
+ * layer shape (split-K slices or the tensor-core kernel's hand-over tiles, which share the space;
+ * per-tile arrival counters and hand-over flags; one status word); 0 for an
  * unsupported shape.  The first W4A8_WORKSPACE_HEADER_BYTES bytes must be zero before the
  * first call (w4a8_workspace_init does that) and are left zero by every call, so one
  * workspace can serve any number of calls that do not overlap on the GPU.
@@ -132,6 +133,8 @@ typedef struct {
     int tile_m;         /* tcgen05: token rows per tile; split-K: 8 x token blocks per CTA (8, 16, 32 or 64) */
     int k_slices;       /* CTAs that share the K range of one tile */
     int ctas;           /* CTAs of the launch */
+    int balanced;       /* tcgen05, more tiles than CTAs: 1 if the tiles x groups units are dealt out evenly, so that
+                           neighbouring CTAs share a tile and hand partial sums over through the workspace */
 } w4a8_plan_info;
 w4a8_status w4a8_plan(int M, int N, int K, int group, w4a8_plan_info* out);
 

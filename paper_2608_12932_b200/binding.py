@@ -197,14 +197,16 @@ def w4a8_gemm_per_channel(qa, sa, packed_w, N, workspace, group=GROUP, out=None,
 
 
 class PlanInfo(ctypes.Structure):
-    _fields_ = [("family", ctypes.c_int), ("tile_m", ctypes.c_int), ("k_slices", ctypes.c_int), ("ctas", ctypes.c_int)]
+    _fields_ = [("family", ctypes.c_int), ("tile_m", ctypes.c_int), ("k_slices", ctypes.c_int), ("ctas", ctypes.c_int),
+                ("balanced", ctypes.c_int)]
 
 
 def w4a8_plan(M, N, K, group=GROUP):
     """What w4a8_gemm would launch for this size on the current device: dict(family, tile_m, k_slices, ctas)."""
     info = PlanInfo()
     _check(lib().w4a8_plan(M, N, K, group, ctypes.byref(info)), "w4a8_plan")
-    return {"family": info.family, "tile_m": info.tile_m, "k_slices": info.k_slices, "ctas": info.ctas}
+    return {"family": info.family, "tile_m": info.tile_m, "k_slices": info.k_slices, "ctas": info.ctas,
+            "balanced": info.balanced}
 
 
 def w4a8_linear(x, packed_w, N, workspace, group=GROUP, out=None, scratch=None, stream=None):

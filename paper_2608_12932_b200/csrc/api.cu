@@ -89,7 +89,8 @@ size_t w4a8_packed_bytes(int N, int K, int group) {
 
 size_t w4a8_workspace_bytes(int M_max, int N, int K, int group) {
     if (!shape_ok(N, K, group) || M_max < 0) return 0;
-    return WS_HEADER_BYTES + slices_bytes(M_max, N, K);
+    const size_t a = slices_bytes(M_max, N, K), b = handover_bytes(M_max, N, K);
+    return WS_HEADER_BYTES + (a > b ? a : b);
 }
 
 w4a8_status w4a8_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
@@ -191,9 +192,10 @@ w4a8_status w4a8_plan(int M, int N, int K, int group, w4a8_plan_info* out) {
         p.tile_m = M <= 8 ? 8 : (M <= 16 ? 16 : (M <= 32 ? 32 : 64));
         p.k_slices = cluster_num_slices(M, N, K);
         p.ctas = tiles * p.k_slices;
+        p.balanced = 0;
     } else {
         p.family = W4A8_PATH_TCGEN05;
-        tcgen05_plan(M, N, K, sms, &p.tile_m, &p.k_slices);
+        tcgen05_plan(M, N, K, sms, &p.tile_m, &p.k_slices, 4, &p.balanced);       // the launcher's own call
         const int all = ((M + p.tile_m - 1) / p.tile_m) * tiles;
         p.ctas = p.k_slices > 1 ? all * p.k_slices : (all < sms ? all : sms);
     }

@@ -76,6 +76,7 @@ constexpr int TMEM_COLS = 512;
 // (cluster launch, two cluster barriers, exchange and reduction of a 208-, 128-, 64-row tile)
 constexpr long TC_FIXED_NS = 4000, TC_GROUP_NS[3] = {650, 540, 440}, TC_SPLIT_NS[3] = {10000, 7000, 4000};
 constexpr int TC_MAX_SPLIT = 4;
+constexpr long TC_BALANCE_NS = 12000;          // balanced walk: hand-over of two partial tiles and a slower pipeline around them
 
 // Shared-memory rings.  The activation tile comes from L2 through TMA with a latency of roughly
 // 2000 cycles, the packed blob from HBM likewise: both rings are deep enough to cover it.
@@ -117,15 +118,18 @@ __device__ __forceinline__ uint32_t sub_zero4(uint32_t q, uint32_t kz) {
 
 // PC ("per channel"): the scales of a channel are the same in every group, so the integer sums of all
 // groups of a tile add up in one accumulator and the tile is drained once (see w4a8_gemm_per_channel).
-template <int TILE_M, bool DEBUG, bool SPLIT, bool PC = false>
+// BAL: balanced walk (see `segment` below).
+template <int TILE_M, bool DEBUG, bool SPLIT, bool PC = false, bool BAL = false>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* __restrict__ packed,
                     const uint16_t* __restrict__ sa, __nv_bfloat16* __restrict__ y,
                     int32_t* __restrict__ debug_partials, uint32_t* __restrict__ status,
-                    int M, int N, int K, int m_tiles, int total_tiles, int S) {
+                    int M, int N, int K, int m_tiles, int total_tiles, int S,
+                    float* __restrict__ handover, uint32_t* __restrict__ handover_flags) {
     using C = Cfg<TILE_M>;
     static_assert(!SPLIT || C::SB * C::B_BYTES >= TILE_M * TILE_N * 4 + 64, "the split-K exchange buffer lives in the activation ring");
     static_assert(!(SPLIT && PC), "the per-channel form is not split along K");
+    static_assert(!BAL || (!SPLIT && !PC), "the balanced walk is for the plain persistent form");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
@@ -179,6 +183,27 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
         mtile = t % m_tiles;
     };
 
+    // The work of a CTA as a list of segments (tile, groups [gb, ge) of it).  Plain persistent walk: whole
+    // tiles unit, unit + num_units, ...  Balanced walk (more tiles than CTAs): the tiles x groups units are
+    // dealt out in equal contiguous ranges, so a CTA's first and last segment may be part of a tile; the CTA
+    // that holds the later groups of such a tile reaches them first (they open its range) and hands its
+    // fp32 sums over through global memory to the CTA that holds the earlier groups (they close its range).
+    const long bal_lo = BAL ? ((long)blockIdx.x * total_tiles * G) / gridDim.x : 0;
+    const long bal_hi = BAL ? ((long)(blockIdx.x + 1) * total_tiles * G) / gridDim.x : 0;
+    auto segment = [&](int idx, int& tile, int& gb, int& ge) -> bool {
+        if (BAL) {
+            tile = (int)(bal_lo / G) + idx;
+            gb = idx == 0 ? (int)(bal_lo % G) : 0;
+            const long left = bal_hi - (long)tile * G;
+            ge = left < G ? (int)left : G;
+            return gb < ge;
+        }
+        tile = unit + idx * num_units;
+        gb = 0;
+        ge = G;
+        return tile < total_tiles;
+    };
+
     bool exchanged = false;                     // SPLIT: this thread has passed the first cluster barrier
     if (warp < 4) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
@@ -186,10 +211,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
             // ------------------------------------------------ producer: activation tiles ----
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = unit; tile < total_tiles && ok; tile += num_units) {
-                int ntile, mtile;
+            for (int si = 0; ok; ++si) {
+                int tile, gb, ge, ntile, mtile;
+                if (!segment(si, tile, gb, ge)) break;
                 tile_of(tile, ntile, mtile);
-                for (int g = 0; g < G; ++g, ++it) {
+                for (int g = gb; g < ge; ++g, ++it) {
                     const uint32_t sb = it % C::SB;
                     if (it >= (uint32_t)C::SB && !(ok = ptx::mbar_wait(done_bar(it - C::SB), done_parity(it - C::SB), abort_flag))) break;
                     ptx::mbar_arrive_expect_tx(bar(B_FULL + sb), C::B_BYTES);
@@ -205,11 +231,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
             // --------------------------------------------------- producer: packed blobs ----
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = unit; tile < total_tiles && ok; tile += num_units) {
-                int ntile, mtile;
+            for (int si = 0; ok; ++si) {
+                int tile, gb, ge, ntile, mtile;
+                if (!segment(si, tile, gb, ge)) break;
                 tile_of(tile, ntile, mtile);
                 const uint8_t* src = packed + ((size_t)ntile * GK + g_lo) * BLOB_BYTES;
-                for (int g = 0; g < G; ++g, ++it) {
+                for (int g = gb; g < ge; ++g, ++it) {
                     const uint32_t sr = it % C::SR, pr = (it / C::SR) & 1;
                     if (!(ok = ptx::mbar_wait(bar(RAW_EMPTY + sr), pr ^ 1, abort_flag))) break;
                     ptx::mbar_arrive_expect_tx(bar(RAW_FULL + sr), BLOB_BYTES);
@@ -234,13 +261,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
             const uint64_t b_desc0 = ptx::smem_desc_k_sw128(smem_base + C::B_OFF);
             uint32_t it = 0, tcount = 0;
             bool ok = true;
-            for (int tile = unit; tile < total_tiles && ok; tile += num_units, ++tcount) {
+            for (int si = 0; ok; ++si, ++tcount) {
+                int tile, gb, ge;
+                if (!segment(si, tile, gb, ge)) break;
                 // PC: both threads add into the buffer of the tile, which the drain warps left zeroed
                 // (integer sums commute, so the order of the two threads' MMAs does not matter)
                 const uint32_t buf = PC ? (tcount & 1u) : par;
                 const uint32_t d_tmem = tmem_base + buf * TILE_M;
                 bool mine = false;
-                for (int g = 0; g < G; ++g, ++it) {
+                for (int g = gb; g < ge; ++g, ++it) {
                     if ((it & 1u) != par) continue;
                     const uint32_t sb = it % C::SB, pb = (it / C::SB) & 1;
                     const uint32_t sa_ = it % C::SA, pas = (it / C::SA) & 1;
@@ -278,8 +307,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
         const uint32_t a_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + C::A_COL0;
         uint32_t it = 0;
         bool ok = true;
-        for (int tile = unit; tile < total_tiles && ok; tile += num_units) {
-            for (int g = 0; g < G; ++g, ++it) {
+        for (int si = 0; ok; ++si) {
+            int tile, gb, ge;
+            if (!segment(si, tile, gb, ge)) break;
+            for (int g = gb; g < ge; ++g, ++it) {
                 const uint32_t sr = it % C::SR, pr = (it / C::SR) & 1;
                 const uint32_t sa_ = it % C::SA;
                 if (!(ok = ptx::mbar_wait(bar(RAW_FULL + sr), pr, abort_flag))) break;
@@ -338,8 +369,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
         }
         uint32_t it = 0, tcount = 0;
         bool ok = true;
-        for (int tile = unit; tile < total_tiles && ok; tile += num_units, ++tcount) {
-            int ntile, mtile;
+        for (int si = 0; ok; ++si, ++tcount) {
+            int tile, gb, ge, ntile, mtile;
+            if (!segment(si, tile, gb, ge)) break;
             tile_of(tile, ntile, mtile);
             const int n = ntile * TILE_N + n_local;
             const int m_base = mtile * TILE_M + h * C::W;
@@ -353,7 +385,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
             for (int i = lane; i < C::W; i += 32)
                 sa_w[i] = (m_base + i < M) ? __half2float(__ushort_as_half(__ldg(sa + m_base + i))) : 0.0f;
             __syncwarp();
-            uint16_t sw_bits = __ldg(reinterpret_cast<const uint16_t*>(sw_ptr));
+            uint16_t sw_bits = __ldg(reinterpret_cast<const uint16_t*>(sw_ptr + (size_t)gb * BLOB_BYTES));
             if (PC) {
                 // one drain per tile: the buffer holds the sum of D over all groups (|sum| < 2^31 for K < 2^13 * 128)
                 const uint32_t buf = tcount & 1u;
@@ -388,10 +420,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                     }
                 }
             }
-            for (int g = 0; g < (PC ? 0 : G); ++g, ++it) {
+            for (int g = gb; g < (PC ? gb : ge); ++g, ++it) {
                 const uint32_t buf = it & 1;
                 const float sw = __half2float(__ushort_as_half(sw_bits));
-                if (g + 1 < G) sw_bits = __ldg(reinterpret_cast<const uint16_t*>(sw_ptr + (size_t)(g + 1) * BLOB_BYTES));
+                if (g + 1 < ge) sw_bits = __ldg(reinterpret_cast<const uint16_t*>(sw_ptr + (size_t)(g + 1) * BLOB_BYTES));
                 if (!(ok = ptx::mbar_wait_hot(done_bar(it), done_parity(it), abort_flag))) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t taddr = lane_taddr + buf * TILE_M;
@@ -424,6 +456,32 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 }
             }
             if (!ok) break;
+            if (BAL && gb > 0) {
+                // Balanced walk: the tile's earlier groups belong to the CTA before this one, which reaches
+                // them at the end of its range.  Hand this CTA's sums over: element (token t, channel n) at
+                // t * 128 + n of this CTA's slot, then the flag (release) once all eight drain warps have written.
+                float* slot = handover + (size_t)blockIdx.x * (TILE_M * TILE_N);
+#pragma unroll
+                for (int i = 0; i < C::W; ++i) __stcg(slot + (size_t)(h * C::W + i) * TILE_N + n_local, facc[i]);
+                __threadfence();
+                ptx::named_bar_sync(2, NUM_DRAIN_WARPS * 32);
+                if (warp == WARP_DRAIN0 && lane == 0) ptx::st_release_gpu_u32(handover_flags + blockIdx.x, 1u);
+                continue;                       // the other CTA stores the tile
+            }
+            if (BAL && ge < G) {
+                // ... and this CTA holds the earlier groups of a tile whose later groups the next CTA summed
+                // long ago (they opened its range): wait for its flag (bounded), add its sums, clear the flag
+                if (warp == WARP_DRAIN0 && lane == 0) {
+                    if (!ptx::wait_flag_acquire_gpu(handover_flags + blockIdx.x + 1, 1u, abort_flag)) ok = false;
+                }
+                ptx::named_bar_sync(2, NUM_DRAIN_WARPS * 32);
+                if (*abort_flag) { ok = false; break; }
+                const float* slot = handover + (size_t)(blockIdx.x + 1) * (TILE_M * TILE_N);
+#pragma unroll
+                for (int i = 0; i < C::W; ++i) facc[i] += __ldcg(slot + (size_t)(h * C::W + i) * TILE_N + n_local);
+                ptx::named_bar_sync(2, NUM_DRAIN_WARPS * 32);
+                if (warp == WARP_DRAIN0 && lane == 0) handover_flags[blockIdx.x + 1] = 0u;     // zero again for the next call
+            }
             if (SPLIT) {
                 // every CTA of the cluster is past its last MMA: the activation rings are free and become
                 // the exchange buffers; push this thread's partials to the CTAs that own them
@@ -498,7 +556,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
     }
 }
 
-template <int TILE_M, bool DEBUG, bool SPLIT, bool PC = false>
+template <int TILE_M, bool DEBUG, bool SPLIT, bool PC = false, bool BAL = false>
 cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed, void* y, int M, int N, int K, int S,
                         void* workspace, int32_t* debug_partials, cudaStream_t stream) {
     using C = Cfg<TILE_M>;
@@ -513,7 +571,7 @@ cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     const int sms = device_sm_count();
     if (!attr_done[dev]) {
-        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT, PC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT, PC, BAL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  C::SMEM_ALLOC);
         if (e != cudaSuccess) return e;
         attr_done[dev] = true;
@@ -523,6 +581,9 @@ cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed
     // persistent: at most one CTA per SM; split-K: one cluster of S CTAs per tile
     const int grid = SPLIT ? total * S : (total < sms ? total : sms);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
+    // BAL: the tiles x groups units are dealt out evenly (a tile may then be shared by two neighbouring
+    // CTAs, which meet through the hand-over area of the workspace); the caller has checked that it applies
+    if (BAL && !(total > grid && grid <= HANDOVER_SLOTS && handover_bytes(M, N, K) > 0)) return cudaErrorInvalidConfiguration;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
     cfg.blockDim = dim3(TC_THREADS, 1, 1);
@@ -535,9 +596,10 @@ cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT, PC>, tmap, static_cast<const uint8_t*>(packed), sa,
+    return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT, PC, BAL>, tmap, static_cast<const uint8_t*>(packed), sa,
                               static_cast<__nv_bfloat16*>(y), debug_partials, reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF),
-                              M, N, K, m_tiles, total, S);
+                              M, N, K, m_tiles, total, S, reinterpret_cast<float*>(ws + WS_HEADER_BYTES),
+                              reinterpret_cast<uint32_t*>(ws + WS_COUNTER_OFF));
 }
 
 // Clusters of S CTAs of the split-K kernel that the device can hold at once (S CTAs need S free SMs
@@ -571,12 +633,17 @@ int max_active_clusters(int S) {
 }
 
 template <bool DEBUG, bool PC = false>
-cudaError_t launch_plan(int tile_m, int S, const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
+cudaError_t launch_plan(int tile_m, int S, bool balanced, const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
                         int M, int N, int K, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
     if (S > 1 && !PC) {
         if (tile_m == 64) return launch_tile<64, DEBUG, true>(qa, sa, packed, y, M, N, K, S, workspace, debug_partials, stream);
         if (tile_m == 128) return launch_tile<128, DEBUG, true>(qa, sa, packed, y, M, N, K, S, workspace, debug_partials, stream);
         return launch_tile<208, DEBUG, true>(qa, sa, packed, y, M, N, K, S, workspace, debug_partials, stream);
+    }
+    if (balanced && !PC) {
+        if (tile_m == 64) return launch_tile<64, DEBUG, false, false, true>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
+        if (tile_m == 128) return launch_tile<128, DEBUG, false, false, true>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
+        return launch_tile<208, DEBUG, false, false, true>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
     }
     if (tile_m == 64) return launch_tile<64, DEBUG, false, PC>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
     if (tile_m == 128) return launch_tile<128, DEBUG, false, PC>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
@@ -591,12 +658,13 @@ cudaError_t launch_plan(int tile_m, int S, const int8_t* qa, const uint16_t* sa,
 // dominates a group, so taller tiles are cheaper per token); a K split into S slices costs
 // TC_SPLIT_NS for the cluster exchange.  Tall tiles win when there are several waves of them, short
 // ones when a tall tiling would leave SMs idle, and a K split when even the shortest tiling does.
-long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split, int max_split) {
+long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split, int max_split, int* balanced) {
     const int heights[3] = {208, 128, 64};
     const int n_tiles = N / TILE_N, G = K / GROUP;
     long best_ns = -1;
     *tile_m = 64;
     *split = 1;
+    if (balanced) *balanced = 0;
     for (int i = 0; i < 3; ++i) {
         if (heights[i] > 64 && M <= heights[i + 1]) continue;        // the next height down already covers M in one tile
         const long tiles = (long)((M + heights[i] - 1) / heights[i]) * n_tiles;
@@ -608,7 +676,16 @@ long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split, int max
                 if (tiles > room) continue;                          // the clusters must all be resident at once
             }
             const long ns = TC_FIXED_NS + waves * TC_GROUP_NS[i] * ((G + S - 1) / S) + (S > 1 ? TC_SPLIT_NS[i] : 0);
-            if (best_ns < 0 || ns < best_ns) { best_ns = ns; *tile_m = heights[i]; *split = S; }   // ties: taller tile, fewer slices
+            if (best_ns < 0 || ns < best_ns) {                        // ties: taller tile, fewer slices
+                best_ns = ns; *tile_m = heights[i]; *split = S;
+                if (balanced) *balanced = 0;
+            }
+            // no split, more tiles than SMs: an even share of all tiles x groups units per CTA, at the price of
+            // handing partial tiles over between neighbours
+            if (S == 1 && balanced && tiles > sms && tiles % sms != 0 && sms <= HANDOVER_SLOTS && handover_bytes(M, N, K) > 0) {
+                const long nb = TC_FIXED_NS + TC_GROUP_NS[i] * ((tiles * G + sms - 1) / sms) + TC_BALANCE_NS;
+                if (nb < best_ns) { best_ns = nb; *tile_m = heights[i]; *split = 1; *balanced = 1; }
+            }
         }
     }
     return best_ns;                                                   // the estimate, for the caller's choice of kernel family
@@ -617,11 +694,11 @@ long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split, int max
 cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
                                 int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream) {
-    int tile_m = 64, S = 1;
-    tcgen05_plan(M, N, K, device_sm_count(), &tile_m, &S, TC_MAX_SPLIT);
+    int tile_m = 64, S = 1, balanced = 0;
+    tcgen05_plan(M, N, K, device_sm_count(), &tile_m, &S, TC_MAX_SPLIT, &balanced);
     if (debug_partials)
-        return launch_plan<true>(tile_m, S, qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
-    return launch_plan<false>(tile_m, S, qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+        return launch_plan<true>(tile_m, S, balanced != 0, qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+    return launch_plan<false>(tile_m, S, balanced != 0, qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
 }
 
 // The same pipeline with one drain per tile: for weights whose scale does not change along K.
@@ -630,10 +707,10 @@ cudaError_t launch_gemm_tcgen05_per_channel(const int8_t* qa, const uint16_t* sa
                                             int M, int N, int K, void* workspace, int32_t* debug_sums,
                                             cudaStream_t stream) {
     int tile_m = 64, S = 1;
-    tcgen05_plan(M, N, K, device_sm_count(), &tile_m, &S, 1);
+    tcgen05_plan(M, N, K, device_sm_count(), &tile_m, &S, 1, nullptr);
     if (debug_sums)
-        return launch_plan<true, true>(tile_m, 1, qa, sa, packed, y, M, N, K, workspace, debug_sums, stream);
-    return launch_plan<false, true>(tile_m, 1, qa, sa, packed, y, M, N, K, workspace, debug_sums, stream);
+        return launch_plan<true, true>(tile_m, 1, false, qa, sa, packed, y, M, N, K, workspace, debug_sums, stream);
+    return launch_plan<false, true>(tile_m, 1, false, qa, sa, packed, y, M, N, K, workspace, debug_sums, stream);
 }
 
 }  // namespace w4a8

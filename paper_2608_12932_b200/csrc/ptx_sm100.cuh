@@ -132,6 +132,28 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// ---- flags in global memory between CTAs of one grid -------------------------------------------
+__device__ __forceinline__ void st_release_gpu_u32(uint32_t* p, uint32_t v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// Polls until *p == want (acquire), the CTA's abort flag is set, or WAIT_LIMIT_NS have passed (it then
+// sets the abort flag).  False if it gave up.
+__device__ __forceinline__ bool wait_flag_acquire_gpu(const uint32_t* p, uint32_t want, volatile uint32_t* abort_flag) {
+    uint64_t t0 = 0;
+    for (uint32_t spin = 1;; ++spin) {
+        uint32_t v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+        if (v == want) return true;
+        if ((spin & 0xFF) == 0) {
+            if (*abort_flag) return false;
+            const uint64_t now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+        }
+        __nanosleep(100);
+    }
+}
+
 // ---- thread-block clusters, distributed shared memory, programmatic dependent launch -----------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;

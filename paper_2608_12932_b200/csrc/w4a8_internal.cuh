@@ -33,6 +33,15 @@ constexpr int WS_STATUS_OFF = 0;
 constexpr int WS_COUNTER_OFF = 256;
 constexpr int WS_HEADER_BYTES = W4A8_WORKSPACE_HEADER_BYTES;
 constexpr int MAX_N_TILES = (WS_HEADER_BYTES - WS_COUNTER_OFF) / 4;   // 960 tiles = N up to 122880
+// Hand-over area of the tcgen05 kernel's balanced walk (after the header, sharing the space of the split-K
+// slices: the two are never in use at once): one fp32 tile of 208 x 128 per CTA; flags in the counter words.
+constexpr int HANDOVER_SLOTS = 192;
+inline size_t handover_bytes(int M, int N, int /*K*/) {
+    // needed where the tcgen05 kernel can run (more than 16 tokens) with more tiles, at its shortest
+    // tiling, than a small sm_100 part has SMs
+    const long tiles = (long)((M + 63) / 64) * (N / TILE_N);
+    return (M > 16 && tiles > 128) ? (size_t)HANDOVER_SLOTS * 208 * TILE_N * sizeof(float) : 0;
+}
 
 // ---- split-K path -----------------------------------------------------------------------------
 constexpr int SPLITK_MAX_M = 64;          // tokens the streaming kernel handles (8 blocks of 8)
@@ -60,8 +69,9 @@ cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void
 cudaError_t launch_gemm_tcgen05_per_channel(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
                                             int M, int N, int K, void* workspace, int32_t* debug_sums,
                                             cudaStream_t stream);
-// tile height and K split (at most max_split slices) the tcgen05 launcher picks; returns its time estimate (ns)
-long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split, int max_split = 4);
+// tile height, K split (at most max_split slices) and, if asked for, whether the balanced walk is taken, as the
+// tcgen05 launcher picks them; returns its time estimate (ns)
+long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split, int max_split = 4, int* balanced = nullptr);
 bool small_m_prefers_tcgen05(int M, int N, int K, int sms);
 
 }  // namespace w4a8

@@ -168,6 +168,22 @@ def test_many_token_tiles_and_very_wide_layer():
     check_case(case, layer, 300, "tcgen05", rows=[0, 1, 207, 208, 299])
 
 
+def test_balanced_walk_hands_partial_tiles_over():
+    """160 tiles of 48 groups on at most 148 CTAs: the launcher deals the 7680 tile-groups out evenly (52 per CTA
+    instead of 96 for the CTAs with two whole tiles), so most tiles are summed by two neighbouring CTAs and
+    meet in the workspace's hand-over area.  Partials bit-exact, output in tolerance, on sampled rows of every
+    token tile; twice, since the hand-over flags must be back at zero for the next call."""
+    case = wl.make_layer(6144, 4096, 41, 1024)
+    layer = DeviceLayer(case, 1024)
+    plan = B.w4a8_plan(1024, 4096, 6144)
+    assert plan["tile_m"] == 208 and plan["balanced"] == 1 and plan["k_slices"] == 1
+    rng = np.random.default_rng(4)
+    rows = np.unique(np.concatenate([[0, 207, 208, 415, 416, 831, 832, 1023], rng.integers(0, 1024, 16)]))
+    y1, _, _ = check_case(case, layer, 1024, "tcgen05", debug=True, rows=rows)
+    y2, _, _ = check_case(case, layer, 1024, "auto", debug=False, rows=rows)
+    assert np.array_equal(y1, y2)
+
+
 def test_persistent_tiles_more_than_sms():
     """160 output tiles over at most 148 CTAs: some CTAs run two tiles back to back."""
     case = wl.make_layer(512, 5120, 33, 1024)
@@ -424,4 +440,6 @@ def test_plan_matches_the_device():
     p = B.w4a8_plan(8, 6144, 4096)
     assert p["family"] == B.PATH_SPLITK and p["ctas"] == 48 * p["k_slices"]
     p = B.w4a8_plan(1024, 24576, 4096)
-    assert p == {"family": B.PATH_TCGEN05, "tile_m": 208, "k_slices": 1, "ctas": sms}
+    assert p == {"family": B.PATH_TCGEN05, "tile_m": 208, "k_slices": 1, "ctas": sms, "balanced": 0}
+    p = B.w4a8_plan(1024, 4096, 12288)                # 160 tiles of 96 groups: evenly dealt out
+    assert p == {"family": B.PATH_TCGEN05, "tile_m": 208, "k_slices": 1, "ctas": sms, "balanced": 1}

@@ -44,7 +44,9 @@ def test_size_queries():
         assert B.w4a8_packed_bytes(N, K) == N * K // 2 + G * N * 5 // 2
         assert B.w4a8_workspace_bytes(0, N, K) == B.WORKSPACE_HEADER_BYTES
         w8, w16, w64, w4096 = (B.w4a8_workspace_bytes(m, N, K) for m in (8, 16, 64, 4096))
-        assert B.WORKSPACE_HEADER_BYTES < w8 < w16 < w64 == w4096
+        assert B.WORKSPACE_HEADER_BYTES < w8 < w16 < w64 <= w4096
+        # from 17 tokens on the tensor-core kernel may need its hand-over area (one fp32 tile per CTA)
+        assert w4096 >= B.WORKSPACE_HEADER_BYTES + 148 * 208 * 128 * 4
         assert (w8 - B.WORKSPACE_HEADER_BYTES) % (8 * N * 4) == 0
     assert B.w4a8_packed_bytes(100, 256) == 0
     assert B.w4a8_packed_bytes(128, 100) == 0
@@ -69,7 +71,7 @@ def test_plan_query_invariants():
                 assert p["family"] == B.PATH_TCGEN05
             if p["family"] == B.PATH_SPLITK:
                 assert p["tile_m"] in (8, 16, 32, 64) and p["tile_m"] >= min(M, 64)
-                assert 1 <= p["k_slices"] <= min(8, G) and p["ctas"] == tiles * p["k_slices"]
+                assert 1 <= p["k_slices"] <= min(8, G) and p["ctas"] == tiles * p["k_slices"] and p["balanced"] == 0
             else:
                 assert p["tile_m"] in (64, 128, 208) and 1 <= p["k_slices"] <= 4
                 all_tiles = -(-M // p["tile_m"]) * tiles
@@ -77,10 +79,17 @@ def test_plan_query_invariants():
                     assert p["ctas"] == all_tiles * p["k_slices"] <= sms and G // p["k_slices"] >= 4
                 else:
                     assert p["ctas"] == min(all_tiles, sms)
+                # the balanced walk only where there are more tiles than CTAs that do not divide evenly, never with a K split
+                assert p["balanced"] in (0, 1)
+                if p["balanced"]:
+                    assert p["k_slices"] == 1 and all_tiles > sms and all_tiles % sms != 0
                 # never a taller tile than the next height down that already covers M
                 assert not (p["tile_m"] == 208 and M <= 128) and not (p["tile_m"] == 128 and M <= 64)
     # several waves of tiles: the tallest tile; a bad shape: an error
     assert B.w4a8_plan(4096, 24576, 4096)["tile_m"] == 208
+    # long K and 160 tiles on 148 SMs: the balanced walk (two rounds of whole tiles would leave most SMs idle half the time)
+    assert B.w4a8_plan(1024, 4096, 12288)["balanced"] == 1
+    assert B.w4a8_plan(4096, 24576, 4096)["balanced"] == 0
     with pytest.raises(B.W4A8Error) as e:
         B.w4a8_plan(8, 100, 256)
     assert e.value.code == B.ERR_SHAPE
