@@ -463,7 +463,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 float* slot = handover + (size_t)blockIdx.x * (TILE_M * TILE_N);
 #pragma unroll
                 for (int i = 0; i < C::W; ++i) __stcg(slot + (size_t)(h * C::W + i) * TILE_N + n_local, facc[i]);
-                __threadfence();
+                // the barrier orders the eight warps' stores before the one release below (cumulative at gpu scope)
                 ptx::named_bar_sync(2, NUM_DRAIN_WARPS * 32);
                 if (warp == WARP_DRAIN0 && lane == 0) ptx::st_release_gpu_u32(handover_flags + blockIdx.x, 1u);
                 continue;                       // the other CTA stores the tile
