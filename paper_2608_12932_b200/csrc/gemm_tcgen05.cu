@@ -76,7 +76,8 @@ constexpr int TMEM_COLS = 512;
 // (cluster launch, two cluster barriers, exchange and reduction of a 208-, 128-, 64-row tile)
 constexpr long TC_FIXED_NS = 4000, TC_GROUP_NS[3] = {650, 540, 440}, TC_SPLIT_NS[3] = {10000, 7000, 4000};
 constexpr int TC_MAX_SPLIT = 4;
-constexpr long TC_BALANCE_NS = 12000;          // balanced walk: hand-over of two partial tiles and a slower pipeline around them
+// balanced walk: hand-over of two partial tiles (208-, 128-, 64-row) and a slower pipeline around them
+constexpr long TC_BALANCE_NS[3] = {12000, 8000, 5000};
 
 // Shared-memory rings.  The activation tile comes from L2 through TMA with a latency of roughly
 // 2000 cycles, the packed blob from HBM likewise: both rings are deep enough to cover it.
@@ -683,7 +684,7 @@ long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split, int max
             // no split, more tiles than SMs: an even share of all tiles x groups units per CTA, at the price of
             // handing partial tiles over between neighbours
             if (S == 1 && balanced && tiles > sms && tiles % sms != 0 && sms <= HANDOVER_SLOTS && handover_bytes(M, N, K) > 0) {
-                const long nb = TC_FIXED_NS + TC_GROUP_NS[i] * ((tiles * G + sms - 1) / sms) + TC_BALANCE_NS;
+                const long nb = TC_FIXED_NS + TC_GROUP_NS[i] * ((tiles * G + sms - 1) / sms) + TC_BALANCE_NS[i];
                 if (nb < best_ns) { best_ns = nb; *tile_m = heights[i]; *split = 1; *balanced = 1; }
             }
         }
