@@ -44,14 +44,14 @@ int device_sm_count() {
 // Between 17 and 64 tokens both kernel families are valid.  Measured on B200 (nanoseconds, cold
 // weights): the streaming kernel costs about 4200 + 570 per group a CTA walks, times the number of
 // CTAs per SM, up to 32 tokens; above, where it walks the token blocks twice, about 7000 + 1140 per
-// group.  The tensor-core kernel's estimate comes from its own planner (tile height, K split).
+// group.  The tensor-core kernel's estimate comes from its own planner (tile height, K split, walk).
 bool small_m_prefers_tcgen05(int M, int N, int K, int sms) {
     if (M <= 16 || M > SPLITK_MAX_M) return M > SPLITK_MAX_M;
     const long G = K / GROUP, tiles = N / TILE_N, S = cluster_num_slices(M, N, K);
     const long groups = ((G + S - 1) / S) * ((tiles * S + sms - 1) / sms);
     const long streaming_ns = M <= 32 ? 4200 + 570 * groups : 7000 + 1140 * groups;
-    int tile_m = 0, split = 0;
-    return tcgen05_plan(M, N, K, sms, &tile_m, &split) < streaming_ns;
+    int tile_m = 0, split = 0, balanced = 0;
+    return tcgen05_plan(M, N, K, sms, &tile_m, &split, 4, &balanced) < streaming_ns;      // as the launcher calls it
 }
 
 }  // namespace w4a8
