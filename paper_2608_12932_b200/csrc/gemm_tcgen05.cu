@@ -370,6 +370,25 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
         }
         uint32_t it = 0, tcount = 0;
         bool ok = true;
+        // token scales (raw fp16 bits) and first group scale of the next segment, requested before the epilogue of
+        // the current one so that their latency is not added to the time the tensor pipe waits for this warp
+        uint16_t next_sa_bits[C::NCH], next_sw_bits = 0;
+        bool have_next = false;
+        auto request = [&](int idx) {
+            int t2, gb2, ge2, nt2, mt2;
+            have_next = segment(idx, t2, gb2, ge2);
+            if (!have_next) return;
+            tile_of(t2, nt2, mt2);
+            const int mb2 = mt2 * TILE_M + h * C::W;
+#pragma unroll
+            for (int k = 0; k < C::NCH; ++k) {
+                const int i = lane + 32 * k;
+                next_sa_bits[k] = (i < C::W && mb2 + i < M) ? __ldg(sa + mb2 + i) : (uint16_t)0;
+            }
+            next_sw_bits = __ldg(reinterpret_cast<const uint16_t*>(packed + ((size_t)nt2 * GK + g_lo + gb2) * BLOB_BYTES +
+                                                                   BLOB_SCALE_OFF + 2 * n_local));
+        };
+        request(0);
         for (int si = 0; ok; ++si, ++tcount) {
             int tile, gb, ge, ntile, mtile;
             if (!segment(si, tile, gb, ge)) break;
@@ -383,10 +402,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
             // this warp's token scales, widened once per tile (rows past M get 0 and are never stored)
             float* sa_w = reinterpret_cast<float*>(smem + C::SA_OFF) + (warp - WARP_DRAIN0) * (C::NCH * 32);
             __syncwarp();
-            for (int i = lane; i < C::W; i += 32)
-                sa_w[i] = (m_base + i < M) ? __half2float(__ushort_as_half(__ldg(sa + m_base + i))) : 0.0f;
+#pragma unroll
+            for (int k = 0; k < C::NCH; ++k)
+                if (lane + 32 * k < C::W) sa_w[lane + 32 * k] = __half2float(__ushort_as_half(next_sa_bits[k]));
             __syncwarp();
-            uint16_t sw_bits = __ldg(reinterpret_cast<const uint16_t*>(sw_ptr + (size_t)gb * BLOB_BYTES));
+            uint16_t sw_bits = next_sw_bits;
             if (PC) {
                 // one drain per tile: the buffer holds the sum of D over all groups (|sum| < 2^31 for K < 2^13 * 128)
                 const uint32_t buf = tcount & 1u;
@@ -457,6 +477,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 }
             }
             if (!ok) break;
+            request(si + 1);
             if (BAL && gb > 0) {
                 // Balanced walk: the tile's earlier groups belong to the CTA before this one, which reaches
                 // them at the end of its range.  Hand this CTA's sums over: element (token t, channel n) at
@@ -506,11 +527,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
             __nv_bfloat16* yrow = y + (size_t)ntile * TILE_N + q * 32 + 8 * (lane & 3);
 #pragma unroll
             for (int b2 = 0; b2 < C::NCH; ++b2) {
+                // The chunk's 32 token scales go to registers first: read one by one between the stores below
+                // they would each wait for the store before them (both are shared-memory accesses the compiler
+                // must keep in order), a chain of 32 round trips per chunk.
+                float sc[32];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const float4 t = *reinterpret_cast<const float4*>(sa_w + b2 * 32 + 4 * k);
+                    sc[4 * k] = t.x; sc[4 * k + 1] = t.y; sc[4 * k + 2] = t.z; sc[4 * k + 3] = t.w;
+                }
                 __syncwarp();
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
                     if (b2 * 32 + i < C::W)
-                        reinterpret_cast<__nv_bfloat16*>(ob + i * 64)[lane] = __float2bfloat16_rn(facc[b2 * 32 + i] * sa_w[b2 * 32 + i]);
+                        reinterpret_cast<__nv_bfloat16*>(ob + i * 64)[lane] = __float2bfloat16_rn(facc[b2 * 32 + i] * sc[i]);
                 __syncwarp();
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
