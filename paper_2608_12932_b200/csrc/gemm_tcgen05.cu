@@ -99,7 +99,7 @@ struct Cfg {
     static constexpr int NCH = (W + 31) / 32;                                 // 32-column chunks per drain warp (the last may be 8 wide)
     static constexpr int LAST = W - 32 * (NCH - 1);                           // width of the last chunk
     static constexpr int SA_OFF = MISC_OFF + 16;   // per drain warp: token scales as fp32
-    static constexpr int OUT_OFF = SA_OFF + NUM_DRAIN_WARPS * NCH * 32 * 4;   // per drain warp: 32 tokens x 32 channels bf16
+    static constexpr int OUT_OFF = (SA_OFF + NUM_DRAIN_WARPS * NCH * 32 * 4 + 127) & ~127;   // per drain warp: 32 tokens x 32 channels bf16 (TMA source: 128-byte aligned)
     static constexpr int SMEM_BYTES = OUT_OFF + NUM_DRAIN_WARPS * 2048;
     static constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;       // slack to align the base to 1024 B
     static_assert(TILE_M == 64 || TILE_M == 128 || TILE_M == 208, "token tile");
@@ -108,7 +108,7 @@ struct Cfg {
     static_assert(SA >= 2 && A_COL0 + SA * A_COLS <= TMEM_COLS, "tensor memory");
     static_assert(SB <= DONE_RING && SA <= DONE_RING, "a stage is freed by the group that used it, at most DONE_RING groups ago");
     static_assert(SMEM_ALLOC <= 227 * 1024, "shared memory");
-    static_assert(OUT_OFF % 16 == 0 && SA_OFF % 16 == 0 && B_BYTES % 1024 == 0, "alignment");
+    static_assert(OUT_OFF % 128 == 0 && SA_OFF % 16 == 0 && B_BYTES % 1024 == 0, "alignment");
 };
 
 __device__ __forceinline__ uint32_t sub_zero4(uint32_t q, uint32_t kz) {
@@ -122,7 +122,8 @@ __device__ __forceinline__ uint32_t sub_zero4(uint32_t q, uint32_t kz) {
 // BAL: balanced walk (see `segment` below).
 template <int TILE_M, bool DEBUG, bool SPLIT, bool PC = false, bool BAL = false>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* __restrict__ packed,
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_constant__ CUtensorMap tmap_y,
+                    const uint8_t* __restrict__ packed,
                     const uint16_t* __restrict__ sa, __nv_bfloat16* __restrict__ y,
                     int32_t* __restrict__ debug_partials, uint32_t* __restrict__ status,
                     int M, int N, int K, int m_tiles, int total_tiles, int S,
@@ -174,6 +175,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
         ptx::tmem_relinquish();
     }
     if (warp == WARP_PRODUCER && lane == 0) ptx::prefetch_tmap(&tmap_qa);
+    if (warp == WARP_DRAIN0 && lane == 0) ptx::prefetch_tmap(&tmap_y);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
@@ -524,6 +526,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
             // stores are 16 bytes per lane along the channel dimension (a thread owns a channel,
             // the output is token-major).  Blocks of up to 32 tokens x this warp's 32 channels.
             uint8_t* ob = smem + C::OUT_OFF + (warp - WARP_DRAIN0) * 2048;
+            const uint32_t ob_addr = smem_base + C::OUT_OFF + (warp - WARP_DRAIN0) * 2048;
             __nv_bfloat16* yrow = y + (size_t)ntile * TILE_N + q * 32 + 8 * (lane & 3);
 #pragma unroll
             for (int b2 = 0; b2 < C::NCH; ++b2) {
@@ -536,15 +539,24 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                     const float4 t = *reinterpret_cast<const float4*>(sa_w + b2 * 32 + 4 * k);
                     sc[4 * k] = t.x; sc[4 * k + 1] = t.y; sc[4 * k + 2] = t.z; sc[4 * k + 3] = t.w;
                 }
+                if (lane == 0) ptx::bulk_wait_group_read0();      // the previous block's TMA store has read `ob`
                 __syncwarp();
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
                     if (b2 * 32 + i < C::W)
                         reinterpret_cast<__nv_bfloat16*>(ob + i * 64)[lane] = __float2bfloat16_rn(facc[b2 * 32 + i] * sc[i]);
-                __syncwarp();
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int row = (lane >> 2) + 8 * i;
+                if (b2 < C::NCH - 1 || C::LAST == 32) {
+                    // a full block of 32 tokens: one TMA store (rows past M are clipped by the map), the warp moves on
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        ptx::tma_store_2d(&tmap_y, ntile * TILE_N + q * 32, m_base + b2 * 32, ob_addr);
+                        ptx::bulk_commit_group();
+                    }
+                } else {
+                    // the 8-token tail of a 208-row tile: 16-byte stores per lane
+                    __syncwarp();
+                    const int row = lane >> 2;
                     const int m = m_base + b2 * 32 + row;
                     if (b2 * 32 + row < C::W && m < M) {
                         const uint4 val = *reinterpret_cast<const uint4*>(ob + row * 64 + 16 * (lane & 3));
@@ -553,6 +565,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint8_t* 
                 }
             }
         }
+        if (lane == 0) ptx::bulk_wait_group0();                   // every tile store of this warp has completed
+        __syncwarp();
     }
 
     if (SPLIT) {
@@ -591,8 +605,10 @@ template <int TILE_M, bool DEBUG, bool SPLIT, bool PC = false, bool BAL = false>
 cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed, void* y, int M, int N, int K, int S,
                         void* workspace, int32_t* debug_partials, cudaStream_t stream) {
     using C = Cfg<TILE_M>;
-    CUtensorMap tmap;
+    CUtensorMap tmap, tmap_y;
     cudaError_t te = make_qa_tensor_map(&tmap, qa, M, K, TILE_M);
+    if (te != cudaSuccess) return te;
+    te = make_y_tensor_map(&tmap_y, y, M, N);
     if (te != cudaSuccess) return te;
 
     int dev = 0;
@@ -627,7 +643,7 @@ cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT, PC, BAL>, tmap, static_cast<const uint8_t*>(packed), sa,
+    return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT, PC, BAL>, tmap, tmap_y, static_cast<const uint8_t*>(packed), sa,
                               static_cast<__nv_bfloat16*>(y), debug_partials, reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF),
                               M, N, K, m_tiles, total, S, reinterpret_cast<float*>(ws + WS_HEADER_BYTES),
                               reinterpret_cast<uint32_t*>(ws + WS_COUNTER_OFF));

@@ -39,4 +39,19 @@ cudaError_t make_qa_tensor_map(CUtensorMap* out, const int8_t* qa, int M, int K,
     return cudaSuccess;
 }
 
+// Map over the bf16 output y[M,N] for the tensor-core kernel's tile stores: boxes of 32 tokens x 32 channels
+// (64 bytes per row), no swizzle; rows past M are not written.
+cudaError_t make_y_tensor_map(CUtensorMap* out, void* y, int M, int N) {
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return cudaErrorNotSupported;
+    const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)N * 2};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    if (encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+    return cudaSuccess;
+}
+
 }  // namespace w4a8

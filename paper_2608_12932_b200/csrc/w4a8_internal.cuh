@@ -49,6 +49,7 @@ constexpr int SPLITK_MAX_GROUPS = 8;      // groups one CTA keeps in shared memo
 int splitk_num_slices(int M, int N, int K);
 
 cudaError_t make_qa_tensor_map(CUtensorMap* out, const int8_t* qa, int M, int K, int box_rows);
+cudaError_t make_y_tensor_map(CUtensorMap* out, void* y, int M, int N);
 cudaError_t launch_quantize_act(const void* x, int M, int K, int8_t* qa, uint16_t* sa, int32_t* asum,
                                 cudaStream_t stream);
 cudaError_t launch_pack_weights(const uint8_t* qw, const uint16_t* scales, const uint8_t* zeros,
