@@ -251,13 +251,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                 const uint64_t t0 = ptx::globaltimer_ns();
                 while (ptx::globaltimer_ns() - t0 < 200000ull) {}
             }
-        } else if ((warp == WARP_MMA || warp == WARP_MMA_ODD) && lane == 0) {
+        } else if (warp == WARP_MMA || warp == WARP_MMA_ODD) {
             // ---------------------------------------------------------------- MMA issuers ----
-            // Two threads, one for the even pipeline steps (accumulator buffer 0) and one for the odd
-            // ones (buffer 1).  A step costs its issuing thread several dependent shared-memory and
-            // tensor-pipe round trips (three barrier probes, four MMAs, a commit); with two threads the
+            // Two warps, one for the even pipeline steps (accumulator buffer 0) and one for the odd
+            // ones (buffer 1).  A step costs its issuer several dependent shared-memory and
+            // tensor-pipe round trips (three barrier probes, four MMAs, a commit); with two issuers the
             // round trips of one step overlap the MMAs of the other.
-            const uint32_t par = (warp == WARP_MMA) ? 0u : 1u;
+            // The whole warp walks the loop and one elected lane issues: with warp-uniform control flow the
+            // MMA operands (addresses, descriptors) are computed once per warp in uniform registers, which
+            // is where the tensor instructions take them from; issued from inside a one-lane branch, every
+            // operand of every MMA went through a register-to-uniform move first.
+            const uint32_t par = __shfl_sync(0xFFFFFFFFu, (warp == WARP_MMA) ? 0u : 1u, 0);
+            const uint32_t tmem_u = __shfl_sync(0xFFFFFFFFu, tmem_base, 0);
             constexpr uint32_t idesc = ptx::idesc_i8(TILE_N, TILE_M, true, true);
             // descriptor of activation stage 0; a stage and a K slice of 32 bytes are plain
             // additions to its (address >> 4) field
@@ -270,7 +275,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                 // PC: both threads add into the buffer of the tile, which the drain warps left zeroed
                 // (integer sums commute, so the order of the two threads' MMAs does not matter)
                 const uint32_t buf = PC ? (tcount & 1u) : par;
-                const uint32_t d_tmem = tmem_base + buf * TILE_M;
+                const uint32_t d_tmem = tmem_u + buf * TILE_M;
                 bool mine = false;
                 for (int g = gb; g < ge; ++g, ++it) {
                     if ((it & 1u) != par) continue;
@@ -281,20 +286,29 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                                                    bar(A_FULL + sa_), pas, abort_flag))) break;
                     ptx::tc_fence_after_sync();
                     const uint64_t bd = b_desc0 + (uint64_t)(sb * (C::B_BYTES / 16));
-                    const uint32_t a_tmem = tmem_base + C::A_COL0 + sa_ * A_COLS;
+                    const uint32_t a_tmem = tmem_u + C::A_COL0 + sa_ * A_COLS;
+                    const uint32_t done = done_bar(it);
+                    if (ptx::elect_one()) {
 #pragma unroll
-                    for (int kk = 0; kk < GROUP / 32; ++kk)       // not PC: the first K slice overwrites the buffer
-                        ptx::mma_i8_ts(d_tmem, a_tmem + 8 * kk, bd + 2 * kk, idesc, (PC || kk) ? 1u : 0u);
-                    ptx::tc_commit(done_bar(it));                 // stages consumed (not PC: accumulator complete)
+                        for (int kk = 0; kk < GROUP / 32; ++kk)   // not PC: the first K slice overwrites the buffer
+                            ptx::mma_i8_ts(d_tmem, a_tmem + 8 * kk, bd + 2 * kk, idesc, (PC || kk) ? 1u : 0u);
+                        ptx::tc_commit(done);                     // stages consumed (not PC: accumulator complete)
+                    }
+                    __syncwarp();
                     mine = true;
                 }
                 if (PC && ok) {
-                    // the tile is complete when the MMAs of both threads are: a commit tracks only its own thread's
-                    if (mine) ptx::tc_commit(bar(TILE_DONE + buf));
-                    else ptx::mbar_arrive(bar(TILE_DONE + buf));
+                    // the tile is complete when the MMAs of both issuers are: a commit tracks only its own thread's
+                    // (elect.sync names the same lane of a full warp every time)
+                    if (ptx::elect_one()) {
+                        if (mine) ptx::tc_commit(bar(TILE_DONE + buf));
+                        else ptx::mbar_arrive(bar(TILE_DONE + buf));
+                    }
+                    __syncwarp();
                 }
             }
-            ptx::tc_commit(bar(FINAL + par));
+            if (ptx::elect_one()) ptx::tc_commit(bar(FINAL + par));
+            __syncwarp();
             // nothing may still be executing on the tensor core when TMEM is freed
             ptx::mbar_wait(bar(FINAL + par), 0, abort_flag);
         }
