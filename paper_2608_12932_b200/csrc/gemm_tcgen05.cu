@@ -282,6 +282,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                     const uint32_t sb = it % C::SB, pb = (it / C::SB) & 1;
                     const uint32_t sa_ = it % C::SA, pas = (it / C::SA) & 1;
                     // accumulator drained; activations landed; weights unpacked
+                    if (TILE_M <= 128) {
+                        // short tiles: the unpacked weights arrive last by far; park on them instead of polling
+                        // (3-4 % at 64..256 tokens), then the other two barriers are there
+                        if (!(ok = ptx::mbar_wait(bar(A_FULL + sa_), pas, abort_flag))) break;
+                        if (!(ok = ptx::mbar_wait(bar(B_FULL + sb), pb, abort_flag))) break;
+                        if (!(ok = ptx::mbar_wait(bar(ACC_EMPTY + buf), ((PC ? tcount : it) >> 1) & 1, abort_flag))) break;
+                    } else
                     if (!(ok = ptx::mbar_wait3_hot(bar(ACC_EMPTY + buf), ((PC ? tcount : it) >> 1) & 1, bar(B_FULL + sb), pb,
                                                    bar(A_FULL + sa_), pas, abort_flag))) break;
                     ptx::tc_fence_after_sync();
@@ -461,7 +468,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                 const uint32_t buf = it & 1;
                 const float sw = __half2float(__ushort_as_half(sw_bits));
                 if (g + 1 < ge) sw_bits = __ldg(reinterpret_cast<const uint16_t*>(sw_ptr + (size_t)(g + 1) * BLOB_BYTES));
-                if (!(ok = ptx::mbar_wait_hot(done_bar(it), done_parity(it), abort_flag))) break;
+                // (short tiles: this warp mostly waits, and a polling loop's probes queue up in front of the unpack
+                // warp's shared-memory accesses on the same scheduler; the parking wait leaves the queue alone)
+                if (!(ok = (TILE_M <= 128 ? ptx::mbar_wait(done_bar(it), done_parity(it), abort_flag)
+                                          : ptx::mbar_wait_hot(done_bar(it), done_parity(it), abort_flag)))) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t taddr = lane_taddr + buf * TILE_M;
                 // All of this warp's columns go to registers with back-to-back loads, then the buffer is
