@@ -282,15 +282,19 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                     const uint32_t sb = it % C::SB, pb = (it / C::SB) & 1;
                     const uint32_t sa_ = it % C::SA, pas = (it / C::SA) & 1;
                     // accumulator drained; activations landed; weights unpacked
+                    // Parking waits, one after the other: polling the three barriers in a loop gained nothing at tall
+                    // tiles (the accumulator hand-back this warp waits for there is 1 000 cycles away) and cost 3-4 %
+                    // at short ones, where the probes queue up in front of the unpack warp's shared-memory accesses
+                    // on the same scheduler.  At short tiles the unpacked weights arrive last by far.
+                    // (Order as measured: weights first at short tiles; activations first at tall ones, 1.5 % there.)
                     if (TILE_M <= 128) {
-                        // short tiles: the unpacked weights arrive last by far; park on them instead of polling
-                        // (3-4 % at 64..256 tokens), then the other two barriers are there
                         if (!(ok = ptx::mbar_wait(bar(A_FULL + sa_), pas, abort_flag))) break;
                         if (!(ok = ptx::mbar_wait(bar(B_FULL + sb), pb, abort_flag))) break;
-                        if (!(ok = ptx::mbar_wait(bar(ACC_EMPTY + buf), ((PC ? tcount : it) >> 1) & 1, abort_flag))) break;
-                    } else
-                    if (!(ok = ptx::mbar_wait3_hot(bar(ACC_EMPTY + buf), ((PC ? tcount : it) >> 1) & 1, bar(B_FULL + sb), pb,
-                                                   bar(A_FULL + sa_), pas, abort_flag))) break;
+                    } else {
+                        if (!(ok = ptx::mbar_wait(bar(B_FULL + sb), pb, abort_flag))) break;
+                        if (!(ok = ptx::mbar_wait(bar(A_FULL + sa_), pas, abort_flag))) break;
+                    }
+                    if (!(ok = ptx::mbar_wait(bar(ACC_EMPTY + buf), ((PC ? tcount : it) >> 1) & 1, abort_flag))) break;
                     ptx::tc_fence_after_sync();
                     const uint64_t bd = b_desc0 + (uint64_t)(sb * (C::B_BYTES / 16));
                     const uint32_t a_tmem = tmem_u + C::A_COL0 + sa_ * A_COLS;

@@ -101,22 +101,6 @@ __device__ __forceinline__ bool mbar_wait_hot(uint32_t bar, uint32_t parity, vol
         }
     }
 }
-// mbar_wait_hot on three barriers at once: the three probes are independent shared-memory round
-// trips, so they overlap instead of costing one latency each
-__device__ __forceinline__ bool mbar_wait3_hot(uint32_t b0, uint32_t p0, uint32_t b1, uint32_t p1, uint32_t b2, uint32_t p2,
-                                               volatile uint32_t* abort_flag) {
-    uint64_t t0 = 0;
-    for (uint32_t spin = 1;; ++spin) {
-        const bool r0 = mbar_test_wait(b0, p0), r1 = mbar_test_wait(b1, p1), r2 = mbar_test_wait(b2, p2);
-        if (r0 && r1 && r2) return true;
-        if ((spin & 0xFFF) == 0) {
-            if (*abort_flag) return false;
-            uint64_t now = globaltimer_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
-        }
-    }
-}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
     uint64_t t0 = 0;
