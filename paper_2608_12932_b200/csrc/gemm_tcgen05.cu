@@ -30,8 +30,10 @@
 //  * there is no accumulator bias / re-arm (which would turn the int->float conversion into an
 //    FMA-pipe add): tcgen05.st traffic to TMEM costs as much port time as tcgen05.ld traffic, more
 //    than the conversion;
-//  * two threads issue the MMAs, one for the even and one for the odd steps: a step costs its issuer
-//    three barrier probes, four MMAs and a commit, each a round trip of about a hundred cycles;
+//  * two warps issue the MMAs, one for the even and one for the odd steps (a step costs its issuer
+//    three barrier waits, four MMAs and a commit); the whole warp walks the loop and an elected lane
+//    issues, which keeps the MMA operands in uniform registers (from inside a one-lane branch every
+//    MMA cost its thread about a hundred cycles of register-to-uniform moves);
 //  * one tcgen05.commit per step, on a ring of "step done" barriers, frees the step's weight and
 //    activation stages and publishes its accumulator.
 //
@@ -42,7 +44,7 @@
 // Warp roles (512 threads, four warpgroups so that setmaxnreg can move registers to the drain:
 // 40 / 40 / 216 / 216 per thread for 208-row tiles, 40 / 96 / 160 / 160 for shorter ones):
 //   warp 0       producer of the activation tiles (2-D TMA loads)
-//   warps 1, 3   MMA issuers (one thread each: even and odd pipeline steps); warp 1 owns TMEM allocation
+//   warps 1, 3   MMA issuers (even and odd pipeline steps; an elected lane issues); warp 1 owns TMEM allocation
 //   warp 2       producer of the packed blobs (1-D bulk copies)
 //   warps 4-7    unpack: raw blob -> signed int8 weight rows in TMEM
 //   warps 8-15   drain: tcgen05.ld -> convert -> FMA with the group scale; final bf16 store
