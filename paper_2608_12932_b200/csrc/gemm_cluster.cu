@@ -133,6 +133,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
     const int r = lane >> 2, j = lane & 3;
     const int set = (warp / WPS) % NSETS;
     const int row0 = (warp % WPS) * (16 * RB) + r;        // block b of this warp: rows row0 + 16b and + 8
+    const int jx = blob_chunk_pos(r, j) * 16;             // chunk j of those rows (they all share the swizzle of r)
 
     if (warp == CL_CONSUMER_WARPS) {
         // ------------------------------------------------------------------ producer ----
@@ -173,8 +174,8 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
 #pragma unroll
             for (int b = 0; b < RB; ++b) {
                 const int row_lo = row0 + 16 * b, row_hi = row_lo + 8;
-                const uint4 wa = *reinterpret_cast<const uint4*>(blob + row_lo * 64 + j * 16);
-                const uint4 wb = *reinterpret_cast<const uint4*>(blob + row_hi * 64 + j * 16);
+                const uint4 wa = *reinterpret_cast<const uint4*>(blob + row_lo * 64 + jx);
+                const uint4 wb = *reinterpret_cast<const uint4*>(blob + row_hi * 64 + jx);
                 const uint32_t wlo[4] = {wa.x, wa.y, wa.z, wa.w}, whi[4] = {wb.x, wb.y, wb.z, wb.w};
                 uint32_t a[4][4];
 #pragma unroll

@@ -98,8 +98,9 @@ gemm_splitk_kernel(const int8_t* __restrict__ qa, const uint16_t* __restrict__ s
         ok = ptx::mbar_wait(ptx::smem_u32(bars + gi), 0, &abort_flag);
         if (!ok) break;
         const uint8_t* blob = blobs + (size_t)gi * BLOB_BYTES;
-        const uint4 wa = *reinterpret_cast<const uint4*>(blob + row_lo * 64 + j * 16);
-        const uint4 wb = *reinterpret_cast<const uint4*>(blob + row_hi * 64 + j * 16);
+        // chunk j of the two rows (rows r and r + 8 share their swizzle)
+        const uint4 wa = *reinterpret_cast<const uint4*>(blob + row_lo * 64 + blob_chunk_pos(row_lo, j) * 16);
+        const uint4 wb = *reinterpret_cast<const uint4*>(blob + row_hi * 64 + blob_chunk_pos(row_lo, j) * 16);
         const uint32_t wlo[4] = {wa.x, wa.y, wa.z, wa.w}, whi[4] = {wb.x, wb.y, wb.z, wb.w};
         uint32_t a[4][4];
 #pragma unroll

@@ -334,6 +334,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
         // One weight row (= one TMEM lane) per thread: 64 packed bytes -> 128 signed bytes -> 32
         // TMEM columns of this group's weight stage, k ascending (4 consecutive k per column).
         const int u = tid - WARP_UNPACK0 * 32;
+        const int sw0 = blob_chunk_pos(u, 0);
         const uint32_t a_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + C::A_COL0;
         uint32_t it = 0;
         bool ok = true;
@@ -347,8 +348,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                 const uint8_t* raw = smem + C::RAW_OFF + sr * RAW_STRIDE;
                 const uint32_t z = (raw[BLOB_ZERO_OFF + (u >> 1)] >> ((u & 1) * 4)) & 0xFu;
                 const uint32_t kz = 0x80808080u - z * 0x01010101u;       // per byte: 0x80 - z, no borrow
+                // chunk p of row u sits at position p ^ ((u >> 1) & 3): eight consecutive rows hit eight bank groups
                 const uint4* rawrow = reinterpret_cast<const uint4*>(raw + u * 64);
-                const uint4 w0 = rawrow[0], w1 = rawrow[1], w2 = rawrow[2], w3 = rawrow[3];
+                const uint4 w0 = rawrow[sw0], w1 = rawrow[sw0 ^ 1], w2 = rawrow[sw0 ^ 2], w3 = rawrow[sw0 ^ 3];
                 // the MMAs that read this stage's previous contents have completed
                 if (it >= (uint32_t)C::SA && !(ok = ptx::mbar_wait(done_bar(it - C::SA), done_parity(it - C::SA), abort_flag))) break;
                 ptx::tc_fence_after_sync();

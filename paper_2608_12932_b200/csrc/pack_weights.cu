@@ -19,7 +19,7 @@ pack_weights_kernel(const uint8_t* __restrict__ qw, const uint16_t* __restrict__
     for (int w = threadIdx.x; w < TILE_N * 16; w += PACK_THREADS) {
         int r = w >> 4, kk = w & 15;
         const uint2 c = *reinterpret_cast<const uint2*>(qw + (size_t)(ntile * TILE_N + r) * K + g * GROUP + kk * 8);
-        words[w] = (c.x & 0x0F0F0F0Fu) | ((c.y & 0x0F0F0F0Fu) << 4);
+        words[r * 16 + blob_chunk_pos(r, kk >> 2) * 4 + (kk & 3)] = (c.x & 0x0F0F0F0Fu) | ((c.y & 0x0F0F0F0Fu) << 4);
     }
     if (threadIdx.x < TILE_N) {
         int r = threadIdx.x;
@@ -42,7 +42,7 @@ unpack_weights_kernel(const uint8_t* __restrict__ packed, int N, int K, uint8_t*
     if (qw) {
         for (int w = threadIdx.x; w < TILE_N * 16; w += PACK_THREADS) {
             int r = w >> 4, kk = w & 15;
-            uint32_t v = words[w];
+            uint32_t v = words[r * 16 + blob_chunk_pos(r, kk >> 2) * 4 + (kk & 3)];
             uint2 c = make_uint2(v & 0x0F0F0F0Fu, (v >> 4) & 0x0F0F0F0Fu);
             *reinterpret_cast<uint2*>(qw + (size_t)(ntile * TILE_N + r) * K + g * GROUP + kk * 8) = c;
         }

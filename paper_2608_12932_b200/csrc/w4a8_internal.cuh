@@ -15,10 +15,16 @@ namespace w4a8 {
 //                 k0 = g*128 + 8*kk: byte b of the word has code[k0+b] in its low nibble and
 //                 code[k0+4+b] in its high nibble, so  w & 0x0F0F0F0F  and  (w>>4) & 0x0F0F0F0F
 //                 are four consecutive-k bytes each, and a 16-byte chunk unpacks to 32 consecutive k.
+//                 The four 16-byte chunks of a row are stored XOR-swizzled: chunk p of row r sits at
+//                 position p ^ ((r >> 1) & 3) of the row (blob_chunk_pos).  A thread-per-row reader
+//                 (16-byte loads at a 64-byte stride) then takes its four chunks without shared-memory
+//                 bank conflicts: eight consecutive rows touch all eight 16-byte bank groups; a
+//                 reader of two rows x four chunks per quarter-warp is conflict-free either way.
 //   [8192, 8448)  128 fp16 scales, row order
 //   [8448, 8512)  128 zero points, two per byte (row 2i low nibble, row 2i+1 high nibble)
 // A blob is exactly the algorithmic 4.15625 bits per weight: no padding.
 constexpr int TILE_N = 128;
+__host__ __device__ constexpr int blob_chunk_pos(int r, int p) { return p ^ ((r >> 1) & 3); }
 constexpr int GROUP = 128;
 constexpr int BLOB_NIBBLE_BYTES = TILE_N * GROUP / 2;        // 8192
 constexpr int BLOB_SCALE_OFF = BLOB_NIBBLE_BYTES;             // 8192
