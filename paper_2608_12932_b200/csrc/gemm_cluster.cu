@@ -159,7 +159,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
         // ----------------------------------------------------------------- consumers ----
         for (int i = tid; i < MP * ng; i += CL_CONSUMER_WARPS * 32) {
             const int m = i / ng, gi = i % ng;
-            asum_s[m * ng_max + gi] = (m < M) ? __ldcg(asum + (size_t)m * G + g0 + gi) : 0;
+            asum_s[gi * MP + m] = (m < M) ? __ldcg(asum + (size_t)m * G + g0 + gi) : 0;      // group-major: see the loads
         }
         ptx::named_bar_sync(1, CL_CONSUMER_WARPS * 32);
         bool ok = true;
@@ -198,7 +198,10 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
                     const uint4 b1 = *reinterpret_cast<const uint4*>(arow + (((2 * j + 1) ^ r) << 4));
                     const uint32_t bq[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
                     const int m0 = 8 * mb + 2 * j;
-                    const int A0 = asum_s[m0 * ng_max + gi], A1 = asum_s[(m0 + 1) * ng_max + gi];
+                    // the two tokens' group sums: one 8-byte load, the four j of a quarter-warp side by side (token-major
+                    // rows of 16 or 32 words put them all into one bank)
+                    const int2 A01 = *reinterpret_cast<const int2*>(asum_s + gi * MP + m0);
+                    const int A0 = A01.x, A1 = A01.y;
                     int d0, d1, d2, d3;       // D = P - z * sum(q_a)
                     if (MB == 2) {
                         // two token blocks give two independent chains: the four MMAs of a block add
