@@ -38,6 +38,8 @@ constexpr int CL_ROW_WARPS = 8;                           // 16 weight rows each
 constexpr int CL_CONSUMER_WARPS = 2 * CL_ROW_WARPS;        // split into warp sets that take groups in turn
 constexpr int CL_THREADS = (CL_CONSUMER_WARPS + 1) * 32;   // + one producer warp
 constexpr int CL_MAX_STAGES = 12;
+constexpr int CL_PART_STRIDE = TILE_N + 4;                 // floats per token row of a partial-sum buffer: the pad spreads the four
+                                                           // token pairs of a warp's store over all banks (a 128-float row puts them in one)
 constexpr int CL_BLOB_STRIDE = 8704;                       // BLOB_BYTES rounded up to a multiple of 128
 constexpr int CL_MAX_S = 8;
 
@@ -55,7 +57,7 @@ __host__ __device__ inline ClLayout cl_layout(int mb, int rb, int stages, int ng
     L.asum_off = L.bar_off + 2 * CL_MAX_STAGES * 8;
     L.red_off = (L.asum_off + 8 * mb * ng_max * 4 + 15) & ~15;
     L.set_off = L.red_off + (8 * mb * (TILE_N / 4) + CL_MAX_S) * 16;   // S slots x ceil(M*32/S) float4
-    L.misc_off = L.set_off + cl_parts(mb, rb) * 8 * mb * TILE_N * 4;   // partial sums, [token][channel] fp32
+    L.misc_off = L.set_off + cl_parts(mb, rb) * 8 * mb * CL_PART_STRIDE * 4;   // partial sums, [token][channel] fp32
     L.total = L.misc_off + 16;
     return L;
 }
@@ -261,14 +263,14 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
                 const int row_lo = row0 + 16 * b, row_hi = row_lo + 8;
 #pragma unroll
                 for (int mb = 0; mb < MB; ++mb) {
-                    float* p = buf + (8 * mb + 2 * j) * TILE_N;
-                    p[row_lo] = facc[b][mb][0]; p[TILE_N + row_lo] = facc[b][mb][1];
-                    p[row_hi] = facc[b][mb][2]; p[TILE_N + row_hi] = facc[b][mb][3];
+                    float* p = buf + (8 * mb + 2 * j) * CL_PART_STRIDE;
+                    p[row_lo] = facc[b][mb][0]; p[CL_PART_STRIDE + row_lo] = facc[b][mb][1];
+                    p[row_hi] = facc[b][mb][2]; p[CL_PART_STRIDE + row_hi] = facc[b][mb][3];
                 }
             }
         };
         if (NPARTS > 1) {
-            put(part + set * (MP * TILE_N));
+            put(part + set * (MP * CL_PART_STRIDE));
         } else {
             if (set == 1) put(part);
             ptx::named_bar_sync(1, CL_CONSUMER_WARPS * 32);
@@ -276,9 +278,9 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
                 const int row_lo = row0, row_hi = row_lo + 8;
 #pragma unroll
                 for (int mb = 0; mb < MB; ++mb) {
-                    const float* p = part + (8 * mb + 2 * j) * TILE_N;
-                    facc[0][mb][0] += p[row_lo]; facc[0][mb][1] += p[TILE_N + row_lo];
-                    facc[0][mb][2] += p[row_hi]; facc[0][mb][3] += p[TILE_N + row_hi];
+                    const float* p = part + (8 * mb + 2 * j) * CL_PART_STRIDE;
+                    facc[0][mb][0] += p[row_lo]; facc[0][mb][1] += p[CL_PART_STRIDE + row_lo];
+                    facc[0][mb][2] += p[row_hi]; facc[0][mb][3] += p[CL_PART_STRIDE + row_hi];
                 }
                 put(part);
             }
@@ -298,10 +300,11 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
     __syncthreads();           // the CTA's partial sums are complete in shared memory
     const float4* part4 = reinterpret_cast<const float4*>(smem + L.set_off);
     auto piece = [&](int q) {
-        float4 v = part4[q];
+        const int q4 = q + (q >> 5);                       // piece q = token q / 32, channels 4 (q % 32)..; rows of 33 float4
+        float4 v = part4[q4];
 #pragma unroll
         for (int p = 1; p < NPARTS; ++p) {                 // set order: deterministic
-            const float4 o = part4[q + p * MP * (TILE_N / 4)];
+            const float4 o = part4[q4 + p * MP * (CL_PART_STRIDE / 4)];
             v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
         }
         return v;
