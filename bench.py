@@ -527,7 +527,7 @@ def run_shape(args):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one split-K GEMM launch at the headline shape,
 # from the ncu capture summarised in profiles/gemm_cluster_qkv_M8.md
-TRAFFIC_BYTES_PER_LAUNCH = 13144064
+TRAFFIC_BYTES_PER_LAUNCH = 13144832
 E2E_DEPTH = int(os.environ.get("W4A8_E2E_DEPTH", "4"))          # host requests in flight in the end-to-end measurement
 
 
