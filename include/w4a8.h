@@ -93,7 +93,7 @@ w4a8_status w4a8_unpack_weights(const void* packed, int N, int K, int group,
                                 void* stream);
 
 /*
- * Per-token dynamic activation quantisation (Sec. 3.4: "8-bit activations").
+ * Per-token dynamic activation quantisation (Sec. 3.4: activations are quantised to 8 bits).
  *   x_bf16  [M,K] row-major, contiguous, 16-byte aligned
  *   qa      [M,K] int8, 16-byte aligned       sa  [M] fp16 bit patterns
  *   asum    [M,K/group] int32 sums of qa over each group (zero-point correction term)
@@ -106,15 +106,21 @@ w4a8_status w4a8_quantize_act(const void* x_bf16, int M, int K, int group,
  * 8-bit activations; Sec. 4: memory-bound for decode-sized M, compute-bound for prefill).
  *   qa, sa, asum     outputs of w4a8_quantize_act (qa 16-byte aligned)
  *   packed_w         output of w4a8_pack_weights for the same N, K, group
- *   y_bf16           [M,N] row-major bf16
+ *   y_bf16           [M,N] row-major bf16, 16-byte aligned (the kernels store it in 8- and 16-byte pieces
+ *                    and through a TMA map; W4A8_ERR_ALIGN otherwise, before anything is enqueued)
  *   workspace        >= w4a8_workspace_bytes(M,N,K,group) bytes, 256-byte aligned, header zeroed once
  *   debug_partials   NULL, or [M,K/group,N] int32 that receives D (slower debug mode)
  * Dispatch: up to 16 tokens the split-K weight-streaming kernel, above 64 the tcgen05 kernel, in
  * between whichever a measured cost model predicts faster for the shape (w4a8_plan tells which).
- * Results are run-to-run deterministic.  The kernels are launched with programmatic stream
- * serialisation: when consecutive library calls share a stream, a kernel may start (and prefetch
- * weights) before its predecessor has finished, and waits on the device before it reads any
- * activation or writes any output.
+ * Results are run-to-run deterministic.
+ * Programmatic dependent launch: w4a8_quantize_act and the weight-streaming kernels for up to 64
+ * tokens are launched with programmatic stream serialisation (the tcgen05 kernel and the workspace
+ * variant of the split-K kernel are launched plainly).  When consecutive library calls share a
+ * stream, such a kernel may start, and prefetch packed weights, before its predecessor in the
+ * stream has finished; it waits on the device before it reads any activation, token scale or group
+ * sum, touches the workspace or writes any output.  packed_w is therefore the one argument that
+ * must be complete before the call is enqueued: do not produce it with a kernel that sits
+ * immediately ahead of the GEMM in the same stream (weights are packed once, offline).
  */
 w4a8_status w4a8_gemm(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
                       const void* packed_w, void* y_bf16,
@@ -170,7 +176,7 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
  * (A single-kernel form, in which the small-M GEMM quantises its own activations, was built and
  * measured slower: every CTA then repeats the row-maximum and division work of the quantiser.)
  *   x_bf16   [M,K] bf16 bits, contiguous, 16-byte aligned
- *   y_bf16   [M,N] bf16 bits, fully overwritten
+ *   y_bf16   [M,N] bf16 bits, 16-byte aligned, fully overwritten
  *   qa, sa, asum   as for w4a8_quantize_act: required scratch, holding the quantised activations afterwards
  * Same shape rules, workspace and status codes as w4a8_gemm.
  */
@@ -187,8 +193,8 @@ w4a8_status w4a8_linear(const void* x_bf16, const void* packed_w, void* y_bf16,
  *   y_host_bf16  HOST [M,N] bf16, valid once `stream` has been synchronised by the caller
  *   x_dev, qa, sa, asum, y_dev   DEVICE staging buffers owned by the caller, sized and aligned
  *                as for w4a8_quantize_act / w4a8_gemm ([M,K] bf16, [M,K] int8, [M] fp16,
- *                [M,K/group] int32, [M,N] bf16)
- * Same shape rules and status codes as w4a8_gemm.
+ *                [M,K/group] int32, [M,N] bf16; x_dev and y_dev 16-byte aligned)
+ * Every argument is checked before the first copy is enqueued.  Same shape rules and status codes as w4a8_gemm.
  */
 w4a8_status w4a8_linear_host(const void* x_host_bf16, void* y_host_bf16,
                              int M, int N, int K, int group, const void* packed_w,
@@ -211,14 +217,19 @@ w4a8_status w4a8_linear_host(const void* x_host_bf16, void* y_host_bf16,
  *   - Calls no cudaMalloc, cudaFree or other allocating routine.  The first call on each device
  *     performs a one-time set-up (it looks up the array's device address and sets a kernel
  *     attribute); make that first call before starting any stream capture.
- *   - All calls on a device share the one array, and each call zeroes the array's header on
- *     `stream` before its kernel: two calls that overlap on the GPU (different streams) race.
- *     Serialise them on one stream.
+ *   - All calls on a device share the one array, and each call zeroes the array's arrival
+ *     counters on `stream` before its kernel: two calls that overlap on the GPU (different
+ *     streams) race.  Serialise them on one stream.
+ *   - y_bf16 needs only 2-byte alignment here (this kernel stores element by element).
+ *   - The status word of this path sits in the array too: w4a8_static_scratch_status reads it
+ *     the way w4a8_check_status reads a workspace's (synchronises `stream`; W4A8_OK, or
+ *     W4A8_ERR_TIMEOUT if a kernel of an earlier call gave up on a bounded wait; clears it).
  */
 #define W4A8_STATIC_SCRATCH_BYTES (4096 + 4 * 1024 * 1024)
 w4a8_status w4a8_gemm_static_scratch(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
                                      const void* packed_w, void* y_bf16,
                                      int M, int N, int K, int group, void* stream);
+w4a8_status w4a8_static_scratch_status(void* stream);
 
 /*
  * Reads back the workspace status word: synchronises `stream`, returns W4A8_OK or

@@ -20,7 +20,7 @@ WORKSPACE_HEADER_BYTES = 4096
 EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w4a8_workspace_init",
            "w4a8_pack_weights", "w4a8_unpack_weights", "w4a8_quantize_act", "w4a8_gemm", "w4a8_gemm_path",
            "w4a8_linear", "w4a8_linear_host", "w4a8_gemm_static_scratch", "w4a8_check_status", "w4a8_plan",
-           "w4a8_gemm_per_channel")
+           "w4a8_gemm_per_channel", "w4a8_static_scratch_status")
 
 _lib = None
 
@@ -70,6 +70,8 @@ def lib():
         L.w4a8_gemm_static_scratch.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp]
         L.w4a8_check_status.restype = ci
         L.w4a8_check_status.argtypes = [vp, vp]
+        L.w4a8_static_scratch_status.restype = ci
+        L.w4a8_static_scratch_status.argtypes = [vp]
         _lib = L
     return _lib
 
@@ -192,7 +194,7 @@ def w4a8_gemm_per_channel(qa, sa, packed_w, N, workspace, group=GROUP, out=None,
         _dev(debug_sums, torch.int32, "debug_sums")
     _check(lib().w4a8_gemm_per_channel(_ptr(qa), _ptr(sa), _ptr(packed_w), _ptr(out), M, N, K, group,
                                        _ptr(workspace), workspace.numel(), _ptr(debug_sums), _stream(stream)),
-           "w4a8_gemm_per_channel")
+           "w4a8_gemm_per_channel", "w4a8_static_scratch_status")
     return out
 
 
@@ -251,6 +253,11 @@ def w4a8_gemm_static_scratch(qa, sa, asum, packed_w, N, group=GROUP, out=None, s
 
 def w4a8_check_status(workspace, stream=None):
     _check(lib().w4a8_check_status(_ptr(workspace), _stream(stream)), "w4a8_check_status")
+
+
+def w4a8_static_scratch_status(stream=None):
+    """The status word of w4a8_gemm_static_scratch's fixed array on the current device (synchronises the stream)."""
+    _check(lib().w4a8_static_scratch_status(_stream(stream)), "w4a8_static_scratch_status")
 
 
 class HostLinear:

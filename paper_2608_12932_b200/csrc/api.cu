@@ -150,8 +150,11 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
     if ((path == W4A8_PATH_SPLITK || path == W4A8_PATH_SPLITK_WORKSPACE) && M > SPLITK_MAX_M) return W4A8_ERR_SHAPE;
     if (M == 0) return W4A8_OK;
     if (!qa || !sa || !asum || !packed_w || !y_bf16 || !workspace) return W4A8_ERR_NULL;
+    // the kernels store y in 8- and 16-byte pieces and through a TMA map (16-byte base); only the
+    // workspace variant of the split-K kernel stores element by element
     if (!aligned(qa, 16) || !aligned(sa, 2) || !aligned(asum, 4) || !aligned(packed_w, 128) ||
-        !aligned(y_bf16, 2) || !aligned(workspace, 256) || (debug_partials && !aligned(debug_partials, 4)))
+        !aligned(y_bf16, path == W4A8_PATH_SPLITK_WORKSPACE ? 2 : 16) || !aligned(workspace, 256) ||
+        (debug_partials && !aligned(debug_partials, 4)))
         return W4A8_ERR_ALIGN;
     if (workspace_bytes < w4a8_workspace_bytes(M, N, K, group)) return W4A8_ERR_WORKSPACE;
     w4a8_status a = arch_check();
@@ -173,7 +176,7 @@ w4a8_status w4a8_gemm_per_channel(const int8_t* qa, const uint16_t* sa, const vo
     if (!shape_ok(N, K, group) || M < 0 || K > (1 << 19)) return W4A8_ERR_SHAPE;    // int32 sums: 15 * 127 * K < 2^31
     if (M == 0) return W4A8_OK;
     if (!qa || !sa || !packed_w || !y_bf16 || !workspace) return W4A8_ERR_NULL;
-    if (!aligned(qa, 16) || !aligned(sa, 2) || !aligned(packed_w, 128) || !aligned(y_bf16, 2) ||
+    if (!aligned(qa, 16) || !aligned(sa, 2) || !aligned(packed_w, 128) || !aligned(y_bf16, 16) ||
         !aligned(workspace, 256) || (debug_sums && !aligned(debug_sums, 4)))
         return W4A8_ERR_ALIGN;
     if (workspace_bytes < w4a8_workspace_bytes(M, N, K, group)) return W4A8_ERR_WORKSPACE;
@@ -218,6 +221,10 @@ w4a8_status w4a8_linear(const void* x_bf16, const void* packed_w, void* y_bf16,
                         void* workspace, size_t workspace_bytes, void* stream) {
     if (!shape_ok(N, K, group) || M < 0) return W4A8_ERR_SHAPE;
     if (M == 0) return W4A8_OK;
+    // everything the second call would refuse is refused before the first one is enqueued
+    if (!x_bf16 || !qa || !sa || !asum || !packed_w || !y_bf16 || !workspace) return W4A8_ERR_NULL;
+    if (!aligned(packed_w, 128) || !aligned(y_bf16, 16) || !aligned(workspace, 256)) return W4A8_ERR_ALIGN;
+    if (workspace_bytes < w4a8_workspace_bytes(M, N, K, group)) return W4A8_ERR_WORKSPACE;
     w4a8_status s = w4a8_quantize_act(x_bf16, M, K, group, qa, sa, asum, stream);
     if (s != W4A8_OK) return s;
     return w4a8_gemm(qa, sa, asum, packed_w, y_bf16, M, N, K, group, workspace, workspace_bytes, nullptr, stream);
@@ -229,7 +236,12 @@ w4a8_status w4a8_linear_host(const void* x_host_bf16, void* y_host_bf16,
                              void* workspace, size_t workspace_bytes, void* stream) {
     if (!shape_ok(N, K, group) || M < 0) return W4A8_ERR_SHAPE;
     if (M == 0) return W4A8_OK;
-    if (!x_host_bf16 || !y_host_bf16 || !x_dev || !y_dev) return W4A8_ERR_NULL;
+    if (!x_host_bf16 || !y_host_bf16 || !x_dev || !y_dev || !qa || !sa || !asum || !packed_w || !workspace)
+        return W4A8_ERR_NULL;
+    if (!aligned(x_dev, 16) || !aligned(qa, 16) || !aligned(sa, 2) || !aligned(asum, 4) || !aligned(packed_w, 128) ||
+        !aligned(y_dev, 16) || !aligned(workspace, 256))
+        return W4A8_ERR_ALIGN;
+    if (workspace_bytes < w4a8_workspace_bytes(M, N, K, group)) return W4A8_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(x_dev, x_host_bf16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return W4A8_ERR_CUDA;
@@ -251,6 +263,12 @@ w4a8_status w4a8_check_status(void* workspace, void* stream) {
     if (cudaMemsetAsync(static_cast<uint8_t*>(workspace) + WS_STATUS_OFF, 0, 4, st) != cudaSuccess) return W4A8_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return W4A8_ERR_CUDA;
     return word == W4A8_ERR_TIMEOUT ? W4A8_ERR_TIMEOUT : W4A8_ERR_CUDA;
+}
+
+w4a8_status w4a8_static_scratch_status(void* stream) {
+    void* scratch = static_scratch_address();        // looks the array's device address up; allocates nothing
+    if (!scratch) return W4A8_ERR_CUDA;
+    return w4a8_check_status(scratch, stream);
 }
 
 }  // extern "C"

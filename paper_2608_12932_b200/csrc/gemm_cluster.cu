@@ -25,7 +25,6 @@
 //    one wave keeps its CTAs under half an SM's shared memory and prefetches as much of its slice
 //    as fits, so that two consecutive launches can be resident together and the weight stream of
 //    the next overlaps the tail of the current one.
-#include <cstdlib>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include "ptx_sm100.cuh"
@@ -416,10 +415,6 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
 // keeps the launch within 0.9 CTAs per SM (clusters of 3 were always slower than 2 or 4).
 int cluster_num_slices(int M, int N, int K) {
     const int G = K / GROUP, tiles = N / TILE_N, sms = device_sm_count();
-    if (const char* e = getenv("W4A8_CLUSTER_S")) {      // tuning aid: force the slice count
-        int v = atoi(e);
-        if (v >= 1 && v <= CL_MAX_S && v <= G) return v;
-    }
     int s;
     // Powers of two only (clusters of other sizes schedule worse).  Up to 8 tokens two CTAs share an
     // SM, so up to 1.75 CTAs per SM still run as one wave; above that one CTA per SM.

@@ -213,11 +213,15 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
     const int G = K / GROUP;
     const int ng_max = (G + S - 1) / S;
     const size_t smem = sk_smem_bytes(MB, ng_max);
-    static bool attr_set = false;      // one attribute per template instance; idempotent
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_splitk_kernel<MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    static bool attr_set[64] = {false};      // function attributes are per device; one array per template instance
+    if (!attr_set[dev]) {
+        e = cudaFuncSetAttribute(gemm_splitk_kernel<MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     gemm_splitk_kernel<MB><<<(N / TILE_N) * S, SK_THREADS, smem, stream>>>(
@@ -276,6 +280,13 @@ void* static_scratch_ptr(int dev, cudaError_t* err) {
     return cached[dev];
 }
 }  // namespace
+
+void* static_scratch_address() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    cudaError_t e = cudaSuccess;
+    return static_scratch_ptr(dev, &e);
+}
 }  // namespace w4a8
 
 extern "C" w4a8_status w4a8_gemm_static_scratch(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
@@ -302,9 +313,11 @@ extern "C" w4a8_status w4a8_gemm_static_scratch(const int8_t* qa, const uint16_t
     void* scratch = static_scratch_ptr(dev, &e);
     if (!scratch) return W4A8_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // the array keeps whatever the previous call left: the header (status word, arrival counters)
-    // must be zero when the kernel starts
-    if (cudaMemsetAsync(scratch, 0, WS_HEADER_BYTES, st) != cudaSuccess) return W4A8_ERR_CUDA;
+    // the array keeps whatever the previous call left: the arrival counters must be zero when the
+    // kernel starts.  The status word ahead of them is left alone, so that a wait that timed out in an
+    // earlier call stays readable (w4a8_check_status with a NULL workspace) until it is read.
+    if (cudaMemsetAsync(static_cast<uint8_t*>(scratch) + WS_COUNTER_OFF, 0, WS_HEADER_BYTES - WS_COUNTER_OFF, st) != cudaSuccess)
+        return W4A8_ERR_CUDA;
     e = launch_gemm_splitk(qa, sa, asum, packed_w, y_bf16, M, N, K, scratch, nullptr, st);
     return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }

@@ -1,8 +1,8 @@
 // Large-M W4A8 GEMM for sm_100a: bulk copies -> shared memory -> int4->int8 unpack into TENSOR
 // MEMORY -> tcgen05.mma kind::i8 (weights from TMEM, activations from shared memory) with int32
 // accumulators in TMEM -> per-group fp32 scaling -> bf16.
-// (Sec. 3.4: "8-bit activations unlock faster INT8 matrix multiplies for the compute-heavy
-// prefill"; Sec. 4: prefill is one long matrix multiplication.)
+// (Sec. 3.4: quantising the activations to 8 bits is what lets the compute-bound prefill run on
+// INT8 tensor cores; Sec. 4: prefill is one long matrix multiplication.)
 //
 // Orientation ("swap-AB"): the 128 output channels of a tile are the MMA's M side (TMEM lanes),
 // the tokens are its N side (TMEM columns).  A drain thread therefore owns ONE output channel:

@@ -1,4 +1,4 @@
-// Per-token dynamic activation quantisation, bf16 -> int8 (Sec. 3.4: "8-bit activations").
+// Per-token dynamic activation quantisation, bf16 -> int8 (Sec. 3.4: activations are quantised to 8 bits).
 //
 // One CTA per token row.  Each thread owns 16-byte chunks (8 bf16) of the row, keeps them
 // in registers across the two passes (absmax, then quantise), so the row is read from

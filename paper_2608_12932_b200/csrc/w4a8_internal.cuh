@@ -65,6 +65,7 @@ cudaError_t launch_unpack_weights(const void* packed, int N, int K, uint8_t* qw,
 cudaError_t launch_gemm_splitk(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
                                void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
                                cudaStream_t stream);
+void* static_scratch_address();              // device address of the static-scratch array on the current device, or NULL
 int device_sm_count();                       // SMs of the current device (cached per device)
 int cluster_num_slices(int M, int N, int K);
 cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,

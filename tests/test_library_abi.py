@@ -131,6 +131,29 @@ def test_shape_validation_needs_no_gpu():
                                ctypes.c_void_p(0x3000), ctypes.c_void_p(0x4000), None) == B.ERR_ALIGN
 
 
+def test_misaligned_output_is_refused_without_a_gpu():
+    """The GEMM kernels store y in 8- and 16-byte pieces, so a bf16 view that starts one element into a
+    buffer must come back as ERR_ALIGN.  Alignment is checked before the device is touched: the pointers
+    below are made-up numbers and nothing is launched."""
+    L = B.lib()
+    vp = ctypes.c_void_p
+    qa, sa, asum, pw, ws = vp(0x10000), vp(0x20000), vp(0x30000), vp(0x40000), vp(0x50000)
+    big = 1 << 30
+    for bad_y in (0x60002, 0x60008):
+        assert L.w4a8_gemm(qa, sa, asum, pw, vp(bad_y), 8, 128, 256, 128, ws, big, None, None) == B.ERR_ALIGN
+        for path in (B.PATH_AUTO, B.PATH_SPLITK, B.PATH_TCGEN05):
+            assert L.w4a8_gemm_path(path, qa, sa, asum, pw, vp(bad_y), 8, 128, 256, 128, ws, big, None, None) == B.ERR_ALIGN
+        assert L.w4a8_gemm_per_channel(qa, sa, pw, vp(bad_y), 8, 128, 256, 128, ws, big, None, None) == B.ERR_ALIGN
+        assert L.w4a8_linear(vp(0x70000), pw, vp(bad_y), 8, 128, 256, 128, qa, sa, asum, ws, big, None) == B.ERR_ALIGN
+        assert L.w4a8_linear_host(vp(0x80000), vp(0x90000), 8, 128, 256, 128, pw, vp(0x70000), qa, sa, asum,
+                                  vp(bad_y), ws, big, None) == B.ERR_ALIGN
+    # the element-by-element kernels take any bf16 pointer: the next check (workspace size) is what refuses this call
+    assert L.w4a8_gemm_path(B.PATH_SPLITK_WORKSPACE, qa, sa, asum, pw, vp(0x60002), 8, 128, 256, 128, ws, 0, None,
+                            None) == B.ERR_WORKSPACE
+    # a misaligned static-scratch call is refused the same way
+    assert L.w4a8_gemm_static_scratch(qa, sa, asum, pw, vp(0x60001), 8, 128, 256, 128, None) == B.ERR_ALIGN
+
+
 def test_missing_library_fails_loudly(tmp_path, monkeypatch):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
