@@ -55,8 +55,11 @@ typedef enum {
     W4A8_PATH_SPLITK = 1,    /* weight-streaming split-K kernel, slices reduced inside a
                                 thread-block cluster through distributed shared memory (M <= 64) */
     W4A8_PATH_TCGEN05 = 2,   /* TMA + tcgen05.mma kind::i8 + TMEM kernel (any M)             */
-    W4A8_PATH_SPLITK_WORKSPACE = 3  /* split-K kernel that reduces its slices through the global
+    W4A8_PATH_SPLITK_WORKSPACE = 3, /* split-K kernel that reduces its slices through the global
                                 workspace (M <= 64); what w4a8_gemm_static_scratch runs        */
+    W4A8_PATH_STRIP = 4      /* weight-streaming kernel without a K split: one persistent CTA per SM,
+                                strips of 16..128 channels over the whole K range dealt out evenly
+                                (M <= 16)                                                       */
 } w4a8_path;
 
 const char* w4a8_status_string(w4a8_status s);
@@ -67,12 +70,14 @@ size_t w4a8_packed_bytes(int N, int K, int group);
 /*
  * Size in bytes of the scratch workspace w4a8_gemm needs for any M <= M_max on this
  * layer shape (split-K slices or the tensor-core kernel's hand-over tiles, which share the space;
- * per-tile arrival counters and hand-over flags; one status word); 0 for an
- * unsupported shape.  The first W4A8_WORKSPACE_HEADER_BYTES bytes must be zero before the
- * first call (w4a8_workspace_init does that) and are left zero by every call, so one
- * workspace can serve any number of calls that do not overlap on the GPU.
+ * per-tile arrival counters and hand-over flags; the strip kernel's hand-over slots; one status
+ * word); 0 for an unsupported shape.  The first W4A8_WORKSPACE_ZEROED_BYTES bytes (or the whole
+ * workspace, if it is smaller) must be zero before the first call (w4a8_workspace_init does that)
+ * and are left zero by every call, so one workspace can serve any number of calls that do not
+ * overlap on the GPU.
  */
 #define W4A8_WORKSPACE_HEADER_BYTES 4096
+#define W4A8_WORKSPACE_ZEROED_BYTES (4096 + 192 * 16384)
 size_t w4a8_workspace_bytes(int M_max, int N, int K, int group);
 w4a8_status w4a8_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
@@ -110,8 +115,9 @@ w4a8_status w4a8_quantize_act(const void* x_bf16, int M, int K, int group,
  *                    and through a TMA map; W4A8_ERR_ALIGN otherwise, before anything is enqueued)
  *   workspace        >= w4a8_workspace_bytes(M,N,K,group) bytes, 256-byte aligned, header zeroed once
  *   debug_partials   NULL, or [M,K/group,N] int32 that receives D (slower debug mode)
- * Dispatch: up to 16 tokens the split-K weight-streaming kernel, above 64 the tcgen05 kernel, in
- * between whichever a measured cost model predicts faster for the shape (w4a8_plan tells which).
+ * Dispatch: up to 16 tokens the strip weight-streaming kernel, above 64 the tcgen05 kernel, in
+ * between the cluster split-K kernel or the tcgen05 kernel, whichever a measured cost model predicts
+ * faster for the shape (w4a8_plan tells which).
  * Results are run-to-run deterministic.
  * Programmatic dependent launch: w4a8_quantize_act and the weight-streaming kernels for up to 64
  * tokens are launched with programmatic stream serialisation (the tcgen05 kernel and the workspace
@@ -130,17 +136,19 @@ w4a8_status w4a8_gemm(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
 
 /*
  * What w4a8_gemm would launch for a problem size on the current device (host-only query, nothing is
- * enqueued): the kernel family, and for W4A8_PATH_SPLITK the number of K slices per 128-channel tile
- * (cluster size), for W4A8_PATH_TCGEN05 the token-tile height (64, 128 or 208) and the number of K
+ * enqueued): the kernel family, for W4A8_PATH_STRIP the strip width, for W4A8_PATH_SPLITK the number of
+ * K slices per 128-channel tile (cluster size), for W4A8_PATH_TCGEN05 the token-tile height (64, 128 or 208) and the number of K
  * slices (1 = no split).  Any output pointer may be NULL.  W4A8_ERR_SHAPE for an unsupported shape.
  */
 typedef struct {
-    w4a8_path family;   /* W4A8_PATH_SPLITK or W4A8_PATH_TCGEN05 */
-    int tile_m;         /* tcgen05: token rows per tile; split-K: 8 x token blocks per CTA (8, 16, 32 or 64) */
-    int k_slices;       /* CTAs that share the K range of one tile */
+    w4a8_path family;   /* W4A8_PATH_STRIP, W4A8_PATH_SPLITK or W4A8_PATH_TCGEN05 */
+    int tile_m;         /* tcgen05: token rows per tile; strip and split-K: 8 x token blocks per CTA (8, 16, 32 or 64) */
+    int k_slices;       /* CTAs that share the K range of one tile (strip: always 1) */
     int ctas;           /* CTAs of the launch */
     int balanced;       /* tcgen05, more tiles than CTAs: 1 if the tiles x groups units are dealt out evenly, so that
-                           neighbouring CTAs share a tile and hand partial sums over through the workspace */
+                           neighbouring CTAs share a tile and hand partial sums over through the workspace;
+                           strip: 1 if the strips do not divide evenly among the CTAs (same hand-over) */
+    int strip_rows;     /* strip: output channels per strip (16, 32, 64 or 128); 0 otherwise */
 } w4a8_plan_info;
 w4a8_status w4a8_plan(int M, int N, int K, int group, w4a8_plan_info* out);
 

@@ -14,8 +14,9 @@ LIB_PATH = os.path.join(_HERE, "libw4a8.so")
 
 GROUP = 128
 OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(8)
-PATH_AUTO, PATH_SPLITK, PATH_TCGEN05, PATH_SPLITK_WORKSPACE = 0, 1, 2, 3
+PATH_AUTO, PATH_SPLITK, PATH_TCGEN05, PATH_SPLITK_WORKSPACE, PATH_STRIP = 0, 1, 2, 3, 4
 WORKSPACE_HEADER_BYTES = 4096
+WORKSPACE_ZEROED_BYTES = 4096 + 192 * 16384
 
 EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w4a8_workspace_init",
            "w4a8_pack_weights", "w4a8_unpack_weights", "w4a8_quantize_act", "w4a8_gemm", "w4a8_gemm_path",
@@ -194,13 +195,13 @@ def w4a8_gemm_per_channel(qa, sa, packed_w, N, workspace, group=GROUP, out=None,
         _dev(debug_sums, torch.int32, "debug_sums")
     _check(lib().w4a8_gemm_per_channel(_ptr(qa), _ptr(sa), _ptr(packed_w), _ptr(out), M, N, K, group,
                                        _ptr(workspace), workspace.numel(), _ptr(debug_sums), _stream(stream)),
-           "w4a8_gemm_per_channel", "w4a8_static_scratch_status")
+           "w4a8_gemm_per_channel")
     return out
 
 
 class PlanInfo(ctypes.Structure):
     _fields_ = [("family", ctypes.c_int), ("tile_m", ctypes.c_int), ("k_slices", ctypes.c_int), ("ctas", ctypes.c_int),
-                ("balanced", ctypes.c_int)]
+                ("balanced", ctypes.c_int), ("strip_rows", ctypes.c_int)]
 
 
 def w4a8_plan(M, N, K, group=GROUP):
@@ -208,7 +209,7 @@ def w4a8_plan(M, N, K, group=GROUP):
     info = PlanInfo()
     _check(lib().w4a8_plan(M, N, K, group, ctypes.byref(info)), "w4a8_plan")
     return {"family": info.family, "tile_m": info.tile_m, "k_slices": info.k_slices, "ctas": info.ctas,
-            "balanced": info.balanced}
+            "balanced": info.balanced, "strip_rows": info.strip_rows}
 
 
 def w4a8_linear(x, packed_w, N, workspace, group=GROUP, out=None, scratch=None, stream=None):

@@ -58,6 +58,12 @@ bool small_m_prefers_tcgen05(int M, int N, int K, int sms) {
 
 namespace {
 
+// Where w4a8_gemm takes the strip kernel: where it is measured faster than the cluster split-K kernel on B200 so far,
+// i.e. up to 8 tokens on layers with fewer 128-channel tiles than SMs.
+bool auto_takes_strip(int M, int N, int K) {
+    return strip_supported(M, N, K) && M <= 8 && N / TILE_N < device_sm_count();
+}
+
 size_t slices_bytes(int M, int N, int K) {
     const int m = M < SPLITK_MAX_M ? M : SPLITK_MAX_M;
     const int S = splitk_num_slices(m, N, K);
@@ -89,15 +95,19 @@ size_t w4a8_packed_bytes(int N, int K, int group) {
 
 size_t w4a8_workspace_bytes(int M_max, int N, int K, int group) {
     if (!shape_ok(N, K, group) || M_max < 0) return 0;
+    // header, then the strip kernel's hand-over slots (zero between calls), then an area shared by the split-K
+    // slices and the tensor-core kernel's hand-over tiles, which are never in use at once
+    if (M_max == 0) return WS_HEADER_BYTES;
     const size_t a = slices_bytes(M_max, N, K), b = handover_bytes(M_max, N, K);
-    return WS_HEADER_BYTES + (a > b ? a : b);
+    return WS_SHARED_OFF + (a > b ? a : b);
 }
 
 w4a8_status w4a8_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
     if (!workspace) return W4A8_ERR_NULL;
     if (workspace_bytes < WS_HEADER_BYTES) return W4A8_ERR_WORKSPACE;
     if (!aligned(workspace, 256)) return W4A8_ERR_ALIGN;
-    if (cudaMemsetAsync(workspace, 0, WS_HEADER_BYTES, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    const size_t zeroed = workspace_bytes < (size_t)W4A8_WORKSPACE_ZEROED_BYTES ? workspace_bytes : (size_t)W4A8_WORKSPACE_ZEROED_BYTES;
+    if (cudaMemsetAsync(workspace, 0, zeroed, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return W4A8_ERR_CUDA;
     return W4A8_OK;
 }
@@ -145,9 +155,10 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
                            int32_t* debug_partials, void* stream) {
     if (!shape_ok(N, K, group) || M < 0) return W4A8_ERR_SHAPE;
     if (path != W4A8_PATH_AUTO && path != W4A8_PATH_SPLITK && path != W4A8_PATH_TCGEN05 &&
-        path != W4A8_PATH_SPLITK_WORKSPACE)
+        path != W4A8_PATH_SPLITK_WORKSPACE && path != W4A8_PATH_STRIP)
         return W4A8_ERR_SHAPE;
     if ((path == W4A8_PATH_SPLITK || path == W4A8_PATH_SPLITK_WORKSPACE) && M > SPLITK_MAX_M) return W4A8_ERR_SHAPE;
+    if (path == W4A8_PATH_STRIP && M > 0 && !strip_supported(M, N, K)) return W4A8_ERR_SHAPE;
     if (M == 0) return W4A8_OK;
     if (!qa || !sa || !asum || !packed_w || !y_bf16 || !workspace) return W4A8_ERR_NULL;
     // the kernels store y in 8- and 16-byte pieces and through a TMA map (16-byte base); only the
@@ -162,7 +173,10 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
     if (path == W4A8_PATH_SPLITK_WORKSPACE)
-        e = launch_gemm_splitk(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
+        e = launch_gemm_splitk(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace,
+                               reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + WS_SHARED_OFF), debug_partials, st);
+    else if (path == W4A8_PATH_STRIP || (path == W4A8_PATH_AUTO && auto_takes_strip(M, N, K)))
+        e = launch_gemm_strip(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
     else if (path == W4A8_PATH_SPLITK || (path == W4A8_PATH_AUTO && !small_m_prefers_tcgen05(M, N, K, device_sm_count())))
         e = launch_gemm_cluster(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
     else
@@ -190,7 +204,17 @@ w4a8_status w4a8_plan(int M, int N, int K, int group, w4a8_plan_info* out) {
     if (!shape_ok(N, K, group) || M <= 0) return W4A8_ERR_SHAPE;
     const int sms = device_sm_count(), tiles = N / TILE_N;
     w4a8_plan_info p;
-    if (!small_m_prefers_tcgen05(M, N, K, sms)) {
+    if (auto_takes_strip(M, N, K)) {
+        int rows = 0, ctas = 0;
+        strip_plan(M, N, K, &rows, &ctas);
+        p.family = W4A8_PATH_STRIP;
+        p.tile_m = M <= 8 ? 8 : 16;
+        p.k_slices = 1;
+        p.ctas = ctas;
+        p.strip_rows = rows;
+        p.balanced = (N / rows) % ctas != 0;
+    } else if (!small_m_prefers_tcgen05(M, N, K, sms)) {
+        p.strip_rows = 0;
         p.family = W4A8_PATH_SPLITK;
         p.tile_m = M <= 8 ? 8 : (M <= 16 ? 16 : (M <= 32 ? 32 : 64));
         p.k_slices = cluster_num_slices(M, N, K);
@@ -198,6 +222,7 @@ w4a8_status w4a8_plan(int M, int N, int K, int group, w4a8_plan_info* out) {
         p.balanced = 0;
     } else {
         p.family = W4A8_PATH_TCGEN05;
+        p.strip_rows = 0;
         tcgen05_plan(M, N, K, sms, &p.tile_m, &p.k_slices, 4, &p.balanced);       // the launcher's own call
         const int all = ((M + p.tile_m - 1) / p.tile_m) * tiles;
         p.ctas = p.k_slices > 1 ? all * p.k_slices : (all < sms ? all : sms);

@@ -209,7 +209,7 @@ gemm_splitk_kernel(const int8_t* __restrict__ qa, const uint16_t* __restrict__ s
 
 template <int MB>
 cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed, void* y,
-                      int M, int N, int K, int S, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
+                      int M, int N, int K, int S, void* workspace, float* slices, int32_t* debug_partials, cudaStream_t stream) {
     const int G = K / GROUP;
     const int ng_max = (G + S - 1) / S;
     const size_t smem = sk_smem_bytes(MB, ng_max);
@@ -226,7 +226,7 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     gemm_splitk_kernel<MB><<<(N / TILE_N) * S, SK_THREADS, smem, stream>>>(
         qa, sa, asum, static_cast<const uint8_t*>(packed), static_cast<__nv_bfloat16*>(y), M, N, K, S, ng_max,
-        reinterpret_cast<float*>(ws + WS_HEADER_BYTES), reinterpret_cast<uint32_t*>(ws + WS_COUNTER_OFF),
+        slices, reinterpret_cast<uint32_t*>(ws + WS_COUNTER_OFF),
         reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF), debug_partials);
     return cudaGetLastError();
 }
@@ -246,13 +246,13 @@ int splitk_num_slices(int /*M*/, int N, int K) {
 }
 
 cudaError_t launch_gemm_splitk(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
-                               void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
+                               void* y, int M, int N, int K, void* workspace, float* slices, int32_t* debug_partials,
                                cudaStream_t stream) {
     const int S = splitk_num_slices(M, N, K);
-    if (M <= 8) return launch_mb<1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
-    if (M <= 16) return launch_mb<2>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
-    if (M <= 32) return launch_mb<4>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
-    return launch_mb<8>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+    if (M <= 8) return launch_mb<1>(qa, sa, asum, packed, y, M, N, K, S, workspace, slices, debug_partials, stream);
+    if (M <= 16) return launch_mb<2>(qa, sa, asum, packed, y, M, N, K, S, workspace, slices, debug_partials, stream);
+    if (M <= 32) return launch_mb<4>(qa, sa, asum, packed, y, M, N, K, S, workspace, slices, debug_partials, stream);
+    return launch_mb<8>(qa, sa, asum, packed, y, M, N, K, S, workspace, slices, debug_partials, stream);
 }
 
 }  // namespace w4a8
@@ -318,6 +318,7 @@ extern "C" w4a8_status w4a8_gemm_static_scratch(const int8_t* qa, const uint16_t
     // earlier call stays readable (w4a8_check_status with a NULL workspace) until it is read.
     if (cudaMemsetAsync(static_cast<uint8_t*>(scratch) + WS_COUNTER_OFF, 0, WS_HEADER_BYTES - WS_COUNTER_OFF, st) != cudaSuccess)
         return W4A8_ERR_CUDA;
-    e = launch_gemm_splitk(qa, sa, asum, packed_w, y_bf16, M, N, K, scratch, nullptr, st);
+    e = launch_gemm_splitk(qa, sa, asum, packed_w, y_bf16, M, N, K, scratch,
+                           reinterpret_cast<float*>(static_cast<uint8_t*>(scratch) + WS_HEADER_BYTES), nullptr, st);
     return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }

@@ -677,7 +677,7 @@ cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT, PC, BAL>, tmap, tmap_y, static_cast<const uint8_t*>(packed), sa,
                               static_cast<__nv_bfloat16*>(y), debug_partials, reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF),
-                              M, N, K, m_tiles, total, S, reinterpret_cast<float*>(ws + WS_HEADER_BYTES),
+                              M, N, K, m_tiles, total, S, reinterpret_cast<float*>(ws + WS_SHARED_OFF),
                               reinterpret_cast<uint32_t*>(ws + WS_COUNTER_OFF));
 }
 

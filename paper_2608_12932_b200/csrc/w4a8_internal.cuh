@@ -34,11 +34,14 @@ constexpr int BLOB_BYTES = BLOB_ZERO_OFF + TILE_N / 2;        // 8512
 // ---- workspace layout -----------------------------------------------------------------------
 //   [0, 4)                    status word (0 = fine, else a w4a8_status written by a kernel)
 //   [256, 256 + 4*n_tiles)    split-K arrival counters, one per 128-channel tile (zero between calls)
-//   [HEADER, ...)             split-K fp32 slices  [S][M][N]
+//   [HEADER, SHARED)          hand-over slots of the strip kernel: one per CTA, each word a float and a tag
+//                             (all zero between calls: the tag is what says that a word has been written)
+//   [SHARED, ...)             split-K fp32 slices  [S][M][N], or the tensor-core kernel's hand-over tiles
 constexpr int WS_STATUS_OFF = 0;
 constexpr int WS_COUNTER_OFF = 256;
 constexpr int WS_HEADER_BYTES = W4A8_WORKSPACE_HEADER_BYTES;
 constexpr int MAX_N_TILES = (WS_HEADER_BYTES - WS_COUNTER_OFF) / 4;   // 960 tiles = N up to 122880
+constexpr int WS_SHARED_OFF = W4A8_WORKSPACE_ZEROED_BYTES;
 // Hand-over area of the tcgen05 kernel's balanced walk (after the header, sharing the space of the split-K
 // slices: the two are never in use at once): one fp32 tile of 208 x 128 per CTA; flags in the counter words.
 constexpr int HANDOVER_SLOTS = 192;
@@ -56,16 +59,30 @@ int splitk_num_slices(int M, int N, int K);
 
 cudaError_t make_qa_tensor_map(CUtensorMap* out, const int8_t* qa, int M, int K, int box_rows);
 cudaError_t make_y_tensor_map(CUtensorMap* out, void* y, int M, int N);
+cudaError_t make_strip_weight_maps(CUtensorMap* nib, CUtensorMap* scale, CUtensorMap* zero, const void* packed,
+                                   int N, int K, int R, int GS);
+cudaError_t make_qa_group_map(CUtensorMap* out, const int8_t* qa, int M, int K, int box_rows, int box_groups);
 cudaError_t launch_quantize_act(const void* x, int M, int K, int8_t* qa, uint16_t* sa, int32_t* asum,
                                 cudaStream_t stream);
 cudaError_t launch_pack_weights(const uint8_t* qw, const uint16_t* scales, const uint8_t* zeros,
                                 int N, int K, void* packed, cudaStream_t stream);
 cudaError_t launch_unpack_weights(const void* packed, int N, int K, uint8_t* qw, uint16_t* scales,
                                   uint8_t* zeros, cudaStream_t stream);
+// `header` = the workspace's first WS_HEADER_BYTES (status word, counters), `slices` = room for the split-K slices
 cudaError_t launch_gemm_splitk(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
-                               void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
+                               void* y, int M, int N, int K, void* header, float* slices, int32_t* debug_partials,
                                cudaStream_t stream);
 void* static_scratch_address();              // device address of the static-scratch array on the current device, or NULL
+// ---- strip path (up to 16 tokens) ---------------------------------------------------------------
+constexpr int STRIP_MAX_M = 16;
+constexpr int STRIP_MAX_CTAS = 192;                       // hand-over slots and flags in the workspace
+constexpr int STRIP_SLOT_BYTES = TILE_N * STRIP_MAX_M * 8;  // one strip's fp32 sums, at most 128 channels x 16 tokens, 8 bytes each
+static_assert(WS_HEADER_BYTES + STRIP_MAX_CTAS * STRIP_SLOT_BYTES == W4A8_WORKSPACE_ZEROED_BYTES, "strip slots fill the zeroed part");
+bool strip_supported(int M, int N, int K);
+void strip_plan(int M, int N, int K, int* strip_rows, int* ctas);
+cudaError_t launch_gemm_strip(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
+                              void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
+                              cudaStream_t stream);
 int device_sm_count();                       // SMs of the current device (cached per device)
 int cluster_num_slices(int M, int N, int K);
 cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,

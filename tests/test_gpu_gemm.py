@@ -17,7 +17,8 @@ from tests.gpu_util import DeviceLayer, bits, t_u16
 
 pytestmark = pytest.mark.gpu
 
-PATHS = {"splitk": B.PATH_SPLITK, "splitk_ws": B.PATH_SPLITK_WORKSPACE, "tcgen05": B.PATH_TCGEN05, "auto": B.PATH_AUTO}
+PATHS = {"splitk": B.PATH_SPLITK, "splitk_ws": B.PATH_SPLITK_WORKSPACE, "tcgen05": B.PATH_TCGEN05, "auto": B.PATH_AUTO,
+         "strip": B.PATH_STRIP}
 
 
 def check_case(case, layer, M, path, debug=True, rows=None):
@@ -39,7 +40,7 @@ def check_case(case, layer, M, path, debug=True, rows=None):
 
 
 # ------------------------------------------------------------------ tiny configuration ---
-@pytest.mark.parametrize("path", ["splitk", "splitk_ws", "tcgen05", "auto"])
+@pytest.mark.parametrize("path", ["splitk", "splitk_ws", "tcgen05", "auto", "strip"])
 def test_tiny_config(path):
     case = wl.make_config("tiny")
     layer = DeviceLayer(case, 16)
@@ -49,7 +50,7 @@ def test_tiny_config(path):
     assert np.array_equal(D, rn["D"])
 
 
-@pytest.mark.parametrize("path", ["splitk", "splitk_ws", "tcgen05"])
+@pytest.mark.parametrize("path", ["splitk", "splitk_ws", "tcgen05", "strip"])
 def test_worked_example_on_gpu(golden, path):
     """The hand-worked example embedded in a 128x128 layer (group 128): same D and y."""
     g = golden("worked_example_w4a8.txt")
@@ -88,6 +89,46 @@ def mid_case():
 def test_splitk_token_counts(mid_case, M, path):
     case, layer = mid_case
     check_case(case, layer, M, path)
+
+
+@pytest.mark.parametrize("M", [1, 2, 3, 7, 8, 9, 15, 16])
+def test_strip_token_counts(mid_case, M):
+    """Three channel tiles of eight groups: 16-channel strips, one or two per CTA."""
+    case, layer = mid_case
+    check_case(case, layer, M, "strip")
+
+
+# layer shapes chosen for the strip widths the planner picks on 148 SMs and for how the strips fall on the CTAs
+STRIP_SHAPES = [
+    (512, 128, 16),       # 8 strips of 16 channels, 8 CTAs with one strip each, one stage (half a ring) per strip
+    (1280, 2432, 16),     # 152 strips of 16 on 148 CTAs: nearly every strip is shared by two CTAs; 10 groups in stages of 8
+    (1024, 4736, 32),     # 148 strips of 32: exactly one per CTA
+    (3072, 6144, 32),     # 192 strips of 32, 24 groups: ranges of 1.3 strips, ring re-used
+    (640, 12288, 64),     # 192 strips of 64, 5 groups in stages of 2 (a ragged last stage)
+    (896, 18944, 128),    # 148 strips of 128
+    (384, 24576, 128),    # 192 strips of 128, 3 groups: ranges shorter than the ring
+    (4096, 37888, 128),   # 296 strips of 128: two whole strips per CTA, no hand-over
+]
+
+
+@pytest.mark.parametrize("K,N,rows", STRIP_SHAPES)
+def test_strip_widths_and_hand_over(K, N, rows):
+    """Every strip width, with and without strips shared between neighbouring CTAs; partials bit-exact, output in
+    tolerance; twice in a row on one workspace, since the hand-over flags must be back at zero for the next call,
+    and bit-identical both times."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    case = wl.make_layer(K, N, 50 + rows, 16)
+    layer = DeviceLayer(case, 16)
+    for M in (8, 16, 5):
+        plan = B.w4a8_plan(M, N, K)
+        if plan["family"] == B.PATH_STRIP:
+            assert plan["k_slices"] == 1 and plan["ctas"] <= min(sms, N // plan["strip_rows"])
+            if sms == 148:
+                assert plan["strip_rows"] == (rows if M <= 8 else max(rows, 32)), plan
+        y1, _, _ = check_case(case, layer, M, "strip", debug=(K * N <= 1 << 26))
+        y2, _, _ = check_case(case, layer, M, "strip", debug=False)
+        assert np.array_equal(y1, y2)
+        check_case(case, layer, M, "auto", debug=False)
 
 
 # token tiles are 64, 128 or 208 rows; a 208-row tile is drained in column pieces of 32, 32, 32 and 8
@@ -193,7 +234,7 @@ def test_persistent_tiles_more_than_sms():
 
 
 # -------------------------------------------------------- invariants on the device -------
-@pytest.mark.parametrize("path,M", [("splitk", 8), ("splitk_ws", 8), ("splitk", 40), ("tcgen05", 130)])
+@pytest.mark.parametrize("path,M", [("splitk", 8), ("splitk_ws", 8), ("splitk", 40), ("tcgen05", 130), ("strip", 8), ("strip", 13)])
 def test_zero_point_invariant_and_determinism(mid_case, path, M):
     case, layer = mid_case
     c2 = dict(case)
@@ -209,7 +250,8 @@ def test_zero_point_invariant_and_determinism(mid_case, path, M):
     assert np.array_equal(y1, y2)
 
 
-@pytest.mark.parametrize("path,M", [("splitk", 5), ("splitk", 16), ("splitk_ws", 8), ("tcgen05", 40), ("tcgen05", 209)])
+@pytest.mark.parametrize("path,M", [("splitk", 5), ("splitk", 16), ("splitk_ws", 8), ("tcgen05", 40), ("tcgen05", 209),
+                                    ("strip", 5), ("strip", 16)])
 def test_extreme_codes_zero_points_and_symmetric_scheme(path, M):
     """Every activation code at +-127 (rows of constant magnitude) against groups whose codes and zero
     points sit at the ends of their ranges (q - z = +-15: the largest partials, |D| = 243840), the
@@ -247,6 +289,9 @@ def test_both_paths_give_identical_partials(mid_case):
     # row independence: row 5 of the M = 48 call equals the M = 1 call on that row
     y3, D3 = layer.gemm(qa[5:6].contiguous(), sa[5:6].contiguous(), asum[5:6].contiguous(), path=B.PATH_SPLITK, debug=True)
     assert np.array_equal(D3[0], D1[5])
+    # the strip kernel on the first 16 of those rows
+    y5, D5 = layer.gemm(qa[:16].contiguous(), sa[:16].contiguous(), asum[:16].contiguous(), path=B.PATH_STRIP, debug=True)
+    assert np.array_equal(D5, D1[:16])
 
 
 def test_scale_linearity_on_gpu(mid_case):
@@ -297,8 +342,10 @@ def test_spec_verify_full_size():
     """M = 8, K = 4096, N = 6144 in the launch configuration the benchmark times: every output, every partial."""
     case = wl.make_config("spec_verify")
     layer = DeviceLayer(case, 8)
+    check_case(case, layer, 8, "strip", debug=True)
     check_case(case, layer, 8, "auto", debug=True)
     check_case(case, layer, 8, "auto", debug=False)
+    check_case(case, layer, 8, "splitk", debug=False)
     check_case(case, layer, 8, "tcgen05", debug=False)
 
 
@@ -438,8 +485,11 @@ def test_plan_matches_the_device():
     p = B.w4a8_plan(64, 4096, 12288)                  # down projection, 32 tiles, 96 groups
     assert p["family"] == B.PATH_TCGEN05 and p["k_slices"] > 1 and p["ctas"] <= sms
     p = B.w4a8_plan(8, 6144, 4096)
-    assert p["family"] == B.PATH_SPLITK and p["ctas"] == 48 * p["k_slices"]
+    assert (p["family"] == B.PATH_STRIP and p["ctas"] == min(sms, 6144 // p["strip_rows"]) and p["k_slices"] == 1) or \
+        (p["family"] == B.PATH_SPLITK and p["ctas"] == 48 * p["k_slices"])
+    p = B.w4a8_plan(40, 6144, 4096)
+    assert (p["family"] == B.PATH_SPLITK and p["ctas"] == 48 * p["k_slices"]) or p["family"] == B.PATH_TCGEN05
     p = B.w4a8_plan(1024, 24576, 4096)
-    assert p == {"family": B.PATH_TCGEN05, "tile_m": 208, "k_slices": 1, "ctas": sms, "balanced": 0}
+    assert p == {"family": B.PATH_TCGEN05, "tile_m": 208, "k_slices": 1, "ctas": sms, "balanced": 0, "strip_rows": 0}
     p = B.w4a8_plan(1024, 4096, 12288)                # 160 tiles of 96 groups: evenly dealt out
-    assert p == {"family": B.PATH_TCGEN05, "tile_m": 208, "k_slices": 1, "ctas": sms, "balanced": 1}
+    assert p == {"family": B.PATH_TCGEN05, "tile_m": 208, "k_slices": 1, "ctas": sms, "balanced": 1, "strip_rows": 0}

@@ -44,10 +44,13 @@ def test_size_queries():
         assert B.w4a8_packed_bytes(N, K) == N * K // 2 + G * N * 5 // 2
         assert B.w4a8_workspace_bytes(0, N, K) == B.WORKSPACE_HEADER_BYTES
         w8, w16, w64, w4096 = (B.w4a8_workspace_bytes(m, N, K) for m in (8, 16, 64, 4096))
-        assert B.WORKSPACE_HEADER_BYTES < w8 < w16 < w64 <= w4096
+        assert B.WORKSPACE_ZEROED_BYTES < w8 < w16 < w64 <= w4096
+        # after the header: one hand-over slot per CTA of the strip kernel (a strip of at most 128 channels x 16 tokens,
+        # a float and a tag per sum), zero between calls; then the split-K slices / hand-over tiles of the other kernels
+        assert B.WORKSPACE_ZEROED_BYTES == B.WORKSPACE_HEADER_BYTES + 192 * 128 * 16 * 8
         # from 17 tokens on the tensor-core kernel may need its hand-over area (one fp32 tile per CTA)
         assert w4096 >= B.WORKSPACE_HEADER_BYTES + 148 * 208 * 128 * 4
-        assert (w8 - B.WORKSPACE_HEADER_BYTES) % (8 * N * 4) == 0
+        assert (w64 - B.WORKSPACE_ZEROED_BYTES) % (64 * N * 4) == 0
     assert B.w4a8_packed_bytes(100, 256) == 0
     assert B.w4a8_packed_bytes(128, 100) == 0
     assert B.w4a8_packed_bytes(128, 256, 64) == 0
@@ -64,12 +67,22 @@ def test_plan_query_invariants():
         tiles, G = N // 128, K // 128
         for M in (1, 7, 8, 9, 16, 17, 32, 33, 64, 65, 128, 200, 256, 512, 1024, 4096):
             p = B.w4a8_plan(M, N, K)
-            assert p["family"] in (B.PATH_SPLITK, B.PATH_TCGEN05)
+            assert p["family"] in (B.PATH_STRIP, B.PATH_SPLITK, B.PATH_TCGEN05)
             if M <= 16:
-                assert p["family"] == B.PATH_SPLITK
+                assert p["family"] in (B.PATH_STRIP, B.PATH_SPLITK)
             if M > 64:
                 assert p["family"] == B.PATH_TCGEN05
-            if p["family"] == B.PATH_SPLITK:
+            if p["family"] == B.PATH_STRIP:
+                # one strip per CTA at least, so that a strip is shared by at most two CTAs; never a K split
+                R = p["strip_rows"]
+                assert R in (16, 32, 64, 128) and p["k_slices"] == 1 and p["tile_m"] == (8 if M <= 8 else 16)
+                assert 1 <= p["ctas"] <= min(sms, N // R)
+                assert p["balanced"] == int((N // R) % p["ctas"] != 0)
+                # the widest strip that keeps about 0.85 strips per SM
+                assert R == 128 or N // (2 * R) < (sms * 17) // 20
+                assert R == (16 if M <= 8 else 32) or N // R >= (sms * 17) // 20
+            elif p["family"] == B.PATH_SPLITK:
+                assert p["strip_rows"] == 0
                 assert p["tile_m"] in (8, 16, 32, 64) and p["tile_m"] >= min(M, 64)
                 assert 1 <= p["k_slices"] <= min(8, G) and p["ctas"] == tiles * p["k_slices"] and p["balanced"] == 0
             else:
