@@ -181,9 +181,9 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
                 uint32_t a[4][4];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    a[q][0] = wlo[q] & 0x0F0F0F0Fu;            // row_lo, k = 32j + 8q + 0..3
+                    a[q][0] = wlo[q] & 0x0F0F0F0Fu;            // row_lo, k = 32j + blob_word_k(q) + 0..3
                     a[q][1] = whi[q] & 0x0F0F0F0Fu;            // row_hi, same k
-                    a[q][2] = (wlo[q] >> 4) & 0x0F0F0F0Fu;     // row_lo, k = 32j + 8q + 4..7
+                    a[q][2] = (wlo[q] >> 4) & 0x0F0F0F0Fu;     // row_lo, eight k further on
                     a[q][3] = (whi[q] >> 4) & 0x0F0F0F0Fu;     // row_hi
                 }
                 const uint16_t* sc = reinterpret_cast<const uint16_t*>(blob + BLOB_SCALE_OFF);
@@ -209,7 +209,8 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
                         // onto one accumulator that starts at the zero-point term (fewer instructions)
                         int c[4] = {-z_lo * A0, -z_lo * A1, -z_hi * A0, -z_hi * A1};
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) mma_u8s8(c, a[q][0], a[q][1], a[q][2], a[q][3], bq[2 * q], bq[2 * q + 1]);
+                        for (int q = 0; q < 4; ++q)
+                            mma_u8s8(c, a[q][0], a[q][1], a[q][2], a[q][3], bq[blob_word_k(q) / 4], bq[blob_word_k(q) / 4 + 2]);
                         d0 = c[0]; d1 = c[1]; d2 = c[2]; d3 = c[3];
                     } else {
                         // four independent MMAs (one per k-step) instead of a dependent chain of four
@@ -217,7 +218,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
                             cq[q][0] = cq[q][1] = cq[q][2] = cq[q][3] = 0;
-                            mma_u8s8(cq[q], a[q][0], a[q][1], a[q][2], a[q][3], bq[2 * q], bq[2 * q + 1]);
+                            mma_u8s8(cq[q], a[q][0], a[q][1], a[q][2], a[q][3], bq[blob_word_k(q) / 4], bq[blob_word_k(q) / 4 + 2]);
                         }
                         int c[4];
 #pragma unroll

@@ -105,9 +105,9 @@ gemm_splitk_kernel(const int8_t* __restrict__ qa, const uint16_t* __restrict__ s
         uint32_t a[4][4];
 #pragma unroll
         for (int s = 0; s < 4; ++s) {
-            a[s][0] = wlo[s] & 0x0F0F0F0Fu;            // row_lo, k = 32j + 8s + 0..3
+            a[s][0] = wlo[s] & 0x0F0F0F0Fu;            // row_lo, k = 32j + blob_word_k(s) + 0..3
             a[s][1] = whi[s] & 0x0F0F0F0Fu;            // row_hi, same k
-            a[s][2] = (wlo[s] >> 4) & 0x0F0F0F0Fu;     // row_lo, k = 32j + 8s + 4..7
+            a[s][2] = (wlo[s] >> 4) & 0x0F0F0F0Fu;     // row_lo, eight k further on
             a[s][3] = (whi[s] >> 4) & 0x0F0F0F0Fu;     // row_hi
         }
         const float s_lo = __half2float(__ushort_as_half(reinterpret_cast<const uint16_t*>(blob + BLOB_SCALE_OFF)[row_lo]));
@@ -122,7 +122,8 @@ gemm_splitk_kernel(const int8_t* __restrict__ qa, const uint16_t* __restrict__ s
             const uint32_t bq[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
             int c[4] = {0, 0, 0, 0};
 #pragma unroll
-            for (int s = 0; s < 4; ++s) mma_u8s8(c, a[s][0], a[s][1], a[s][2], a[s][3], bq[2 * s], bq[2 * s + 1]);
+            for (int s = 0; s < 4; ++s)
+                mma_u8s8(c, a[s][0], a[s][1], a[s][2], a[s][3], bq[blob_word_k(s) / 4], bq[blob_word_k(s) / 4 + 2]);
             const int m0 = 8 * mb + 2 * j;
             const int A0 = asum_s[m0 * ng_max + gi], A1 = asum_s[(m0 + 1) * ng_max + gi];
             const int d0 = c[0] - z_lo * A0, d1 = c[1] - z_lo * A1;

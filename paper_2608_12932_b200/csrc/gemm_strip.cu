@@ -25,8 +25,9 @@
 //    own last strip is still being multiplied (bounded retries), zeroes them for the next call,
 //    adds (earlier + later groups: a fixed order) and stores the strip.  Every SM thus streams the
 //    same number of bytes, whatever the layer's width.
-//  * Consumers: eight warps, each with two of a stage's sixteen units (the same 16 rows of two groups), whose
-//    loads and MMAs interleave.  mma.sync m16n8k32 (u8 x s8 -> s32), weights as the 16-row operand.  The low nibbles
+//  * Consumers: eight warps, each with two of a stage's sixteen units, whose loads and MMAs interleave: two
+//    16-row blocks of one group (they share the activation fragments), or, in 16-row strips, the one block of
+//    two groups.  mma.sync m16n8k32 (u8 x s8 -> s32), weights as the 16-row operand.  The low nibbles
 //    feed one chain of two MMAs that starts at the zero-point term -z * sum(q_a), the high nibbles -
 //    masked in place, i.e. as 16 x code - a second chain; D = low + high / 16 exactly (int32), scaled
 //    by the group scale in fp32.  A warp keeps its sums over the groups it meets in registers; at the
@@ -76,11 +77,20 @@ __host__ __device__ inline StLayout st_layout(int mb, int rblk, int stages, int 
     L.asum_off = (L.bar_off + (2 * ST_MAX_STAGES + 2) * 8 + 15) & ~15;
     L.sa_off = L.asum_off + G * mp * 4;                     // group sums, [group][token]
     L.part_off = (L.sa_off + mp * 4 + 15) & ~15;            // token scales as fp32
-    L.take_off = L.part_off + ST_CONSUMER_WARPS * mb * 32 * 16;   // one float4 per consumer lane and token block
+    L.take_off = L.part_off + ST_CONSUMER_WARPS * (rblk >= 2 ? 2 : 1) * mb * 32 * 16;   // one float4 per consumer lane, row block and token block
     L.ystage_off = L.take_off + rblk * mb * 32 * 16;        // the neighbour's sums of a shared strip
     L.misc_off = L.ystage_off + mp * (32 * rblk + 16);      // a strip's bf16 outputs, [token][channel], rows padded by 16 B
     L.total = L.misc_off + 16;
     return L;
+}
+
+// the same with a zero accumulator going in (no registers to clear)
+__device__ __forceinline__ void mma_u8s8_z(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                           uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
 }
 
 __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -271,22 +281,33 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
         }
         ptx::named_bar_sync(1, ST_CONSUMER_WARPS * 32);
 
-        // the warp's two units of a stage: 16-row block rb of groups gi and gi + GS / 2
+        // The warp's two units of a stage.  SHARE (strips of 32 rows and more): two 16-row blocks, rows 32 rp ..
+        // 32 rp + 31, of ONE group gi - the activation fragments and group sums are loaded once for both.
+        // Strips of 16 rows: the one block of groups gi and gi + GS / 2.
+        constexpr bool SHARE = RBLK >= 2;
+        constexpr int NF = SHARE ? 2 : 1;                    // row blocks a lane accumulates
+        constexpr int WPG = SHARE ? RBLK / 2 : 1;            // warps per group
         constexpr int HALF_GS = GS / 2;
-        const int rb = warp % RBLK, gi = warp / RBLK;
+        const int gi = warp / WPG, rp = warp % WPG;
         const int r = lane >> 2, j = lane & 3;
-        const int row = rb * 16 + r;                         // row inside the strip; row + 8 is the lane's second row
-        // per-lane offsets inside a stage, for the first unit; the second unit's differ by compile-time constants
-        const uint32_t nib_off = gi * NIB_G + row * 64 + blob_chunk_pos(r, j) * 16;   // rows r and r + 8 share their swizzle
+        const int row = rp * (SHARE ? 32 : 16) + r;          // first unit's row inside the strip (its second row is + 8)
+        // second unit relative to the first, in bytes inside a stage
+        constexpr uint32_t U1_NIB = SHARE ? 16 * 64 : HALF_GS * NIB_G, U1_SC = SHARE ? 32 : HALF_GS * SC_G;
+        constexpr uint32_t U1_Z = SHARE ? 8 : HALF_GS * Z_G, U1_ACT = SHARE ? 0 : HALF_GS * MP * GROUP;
+        constexpr uint32_t U1_ASUM = SHARE ? 0 : HALF_GS * MP * 4;
+        // per-lane offsets inside a stage, first unit
+        const uint32_t nib_off = gi * NIB_G + row * 64 + blob_chunk_pos(r, j) * 16;   // rows r, r + 8, r + 16, r + 24 share their swizzle
         const uint32_t sc_off = SC_BASE + gi * SC_G + 2 * row;
         const uint32_t z_off = Z_BASE + gi * Z_G + (row >> 1);
         const int zsh = (r & 1) * 4;
         const uint32_t b0_off = ST_W_BYTES + gi * (MP * GROUP) + r * 128 + (((2 * j) ^ r) << 4);   // chunk 2j of the token row; 2j + 1 is ^ 16
         const uint32_t asum_lane = smem_base + L.asum_off + (gi * MP + 2 * j) * 4;
-        const uint32_t part_lane = smem_base + L.part_off + (warp * MB * 32 + lane) * 16;
-        float facc[MB][4];
+        const uint32_t part_lane = smem_base + L.part_off + (warp * NF * MB * 32 + lane) * 16;
+        float facc[NF][MB][4];
 #pragma unroll
-        for (int mb = 0; mb < MB; ++mb) facc[mb][0] = facc[mb][1] = facc[mb][2] = facc[mb][3] = 0.0f;
+        for (int f = 0; f < NF; ++f)
+#pragma unroll
+            for (int mb = 0; mb < MB; ++mb) facc[f][mb][0] = facc[f][mb][1] = facc[f][mb][2] = facc[f][mb][3] = 0.0f;
 
         bool ok = true;
         int flushed = 0;                                     // strips of this CTA flushed so far
@@ -295,12 +316,15 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
             if (flushed > 0) ok = ok && st_wait(part_empty, (uint32_t)((flushed - 1) & 1), abort_flag);
             if (ok) {
 #pragma unroll
-                for (int mb = 0; mb < MB; ++mb) {
-                    // the high-nibble chain carried 16 x code: the sums are 16 x D, a power of two taken out here
-                    ptx::sts128(part_lane + mb * 512,
-                                make_float4(facc[mb][0] * 0.0625f, facc[mb][1] * 0.0625f, facc[mb][2] * 0.0625f, facc[mb][3] * 0.0625f));
-                    facc[mb][0] = facc[mb][1] = facc[mb][2] = facc[mb][3] = 0.0f;
-                }
+                for (int f = 0; f < NF; ++f)
+#pragma unroll
+                    for (int mb = 0; mb < MB; ++mb) {
+                        // the high-nibble chain carried 16 x code: the sums are 16 x D, a power of two taken out here
+                        ptx::sts128(part_lane + (f * MB + mb) * 512,
+                                    make_float4(facc[f][mb][0] * 0.0625f, facc[f][mb][1] * 0.0625f, facc[f][mb][2] * 0.0625f,
+                                                facc[f][mb][3] * 0.0625f));
+                        facc[f][mb][0] = facc[f][mb][1] = facc[f][mb][2] = facc[f][mb][3] = 0.0f;
+                    }
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(part_full);
             }
@@ -320,76 +344,94 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
             if (tid == 0 && i < 40) ST_STAMP(16 + i);
 #if !defined(ST_ABL) || ST_ABL != 1
             {
-                const int g0 = sg * GS + gi, g1 = g0 + HALF_GS;
+                const int g0 = sg * GS + gi, g1 = SHARE ? g0 : g0 + HALF_GS;
                 // narrow strips of 16 rows fetch the zero points of 32 rows: the odd strip's are the second half
                 const uint32_t zo = stage + z_off + ((R == 16 && (strip & 1)) ? 8 : 0);
                 const uint4 wa0 = ptx::lds128(stage + nib_off), wb0 = ptx::lds128(stage + nib_off + 8 * 64);
-                const uint4 wa1 = ptx::lds128(stage + nib_off + HALF_GS * NIB_G), wb1 = ptx::lds128(stage + nib_off + HALF_GS * NIB_G + 8 * 64);
+                const uint4 wa1 = ptx::lds128(stage + nib_off + U1_NIB), wb1 = ptx::lds128(stage + nib_off + U1_NIB + 8 * 64);
                 float s_lo0 = __half2float(__ushort_as_half((unsigned short)ptx::lds_u16(stage + sc_off)));
                 float s_hi0 = __half2float(__ushort_as_half((unsigned short)ptx::lds_u16(stage + sc_off + 16)));
-                float s_lo1 = __half2float(__ushort_as_half((unsigned short)ptx::lds_u16(stage + sc_off + HALF_GS * SC_G)));
-                float s_hi1 = __half2float(__ushort_as_half((unsigned short)ptx::lds_u16(stage + sc_off + HALF_GS * SC_G + 16)));
+                float s_lo1 = __half2float(__ushort_as_half((unsigned short)ptx::lds_u16(stage + sc_off + U1_SC)));
+                float s_hi1 = __half2float(__ushort_as_half((unsigned short)ptx::lds_u16(stage + sc_off + U1_SC + 16)));
                 const int z_lo0 = (ptx::lds_u8(zo) >> zsh) & 0xF, z_hi0 = (ptx::lds_u8(zo + 4) >> zsh) & 0xF;
-                const int z_lo1 = (ptx::lds_u8(zo + HALF_GS * Z_G) >> zsh) & 0xF, z_hi1 = (ptx::lds_u8(zo + HALF_GS * Z_G + 4) >> zsh) & 0xF;
+                const int z_lo1 = (ptx::lds_u8(zo + U1_Z) >> zsh) & 0xF, z_hi1 = (ptx::lds_u8(zo + U1_Z + 4) >> zsh) & 0xF;
                 // groups past the end of K (a ragged last stage): whatever the slot holds there must add nothing
                 if (g0 >= G) s_lo0 = s_hi0 = 0.0f;
                 if (g1 >= G) s_lo1 = s_hi1 = 0.0f;
                 const uint32_t asum_g = asum_lane + sg * (GS * MP * 4);
+                constexpr uint32_t LO = 0x0F0F0F0Fu, HI = 0xF0F0F0F0u;
 #pragma unroll
                 for (int mb = 0; mb < MB; ++mb) {
                     // token row 8*mb + r of a group's tile: 128 B, 16-byte chunks XOR-swizzled by the row index
                     const uint32_t ab = stage + b0_off + mb * 1024;
                     const uint4 p0 = ptx::lds128(ab), p1 = ptx::lds128(ab ^ 16u);
-                    const uint4 q0 = ptx::lds128(ab + HALF_GS * MP * GROUP), q1 = ptx::lds128((ab + HALF_GS * MP * GROUP) ^ 16u);
                     const uint2 A0 = ptx::lds64(asum_g + mb * 32);                        // the two tokens' group sums
-                    const uint2 A1 = ptx::lds64(asum_g + HALF_GS * MP * 4 + mb * 32);
+                    uint4 q0 = p0, q1 = p1;
+                    uint2 A1 = A0;
+                    if (!SHARE) {
+                        q0 = ptx::lds128(ab + U1_ACT);
+                        q1 = ptx::lds128((ab + U1_ACT) ^ 16u);
+                        A1 = ptx::lds64(asum_g + U1_ASUM + mb * 32);
+                    }
                     int cl0[4] = {-z_lo0 * (int)A0.x, -z_lo0 * (int)A0.y, -z_hi0 * (int)A0.x, -z_hi0 * (int)A0.y};
                     int cl1[4] = {-z_lo1 * (int)A1.x, -z_lo1 * (int)A1.y, -z_hi1 * (int)A1.x, -z_hi1 * (int)A1.y};
-                    int ch0[4] = {0, 0, 0, 0}, ch1[4] = {0, 0, 0, 0};
-                    // low nibbles: k = 32j + 8q + 0..3 of word q, paired with activation word 2q; high nibbles, left in
-                    // place (16 x code): k = 32j + 8q + 4..7, paired with activation word 2q + 1
+                    int ch0[4], ch1[4];
+                    // Words x, y of a packed chunk carry the runs of four k (a0, a2) and (a1, a3) in their (low, high)
+                    // nibbles, words z, w the runs (a4, a6) and (a5, a7): the low nibbles of a word pair go with
+                    // activation words (0, 1) or (4, 5), the high ones - left in place, i.e. 16 x code - with (2, 3) or (6, 7).
 #if defined(ST_ABL) && ST_ABL == 2
-                    cl0[0] += wa0.x + p0.x; cl1[0] += wa1.x + q0.x; ch0[0] += wb0.y + p1.y; ch1[0] += wb1.y + q1.y;
+                    cl0[0] += wa0.x + p0.x; cl1[0] += wa1.x + q0.x; ch0[0] = ch0[1] = ch0[2] = ch0[3] = wb0.y + p1.y; ch1[0] = ch1[1] = ch1[2] = ch1[3] = wb1.y + q1.y;
 #else
-                    mma_u8s8(cl0, wa0.x & 0x0F0F0F0Fu, wb0.x & 0x0F0F0F0Fu, wa0.y & 0x0F0F0F0Fu, wb0.y & 0x0F0F0F0Fu, p0.x, p0.z);
-                    mma_u8s8(cl1, wa1.x & 0x0F0F0F0Fu, wb1.x & 0x0F0F0F0Fu, wa1.y & 0x0F0F0F0Fu, wb1.y & 0x0F0F0F0Fu, q0.x, q0.z);
-                    mma_u8s8(ch0, wa0.x & 0xF0F0F0F0u, wb0.x & 0xF0F0F0F0u, wa0.y & 0xF0F0F0F0u, wb0.y & 0xF0F0F0F0u, p0.y, p0.w);
-                    mma_u8s8(ch1, wa1.x & 0xF0F0F0F0u, wb1.x & 0xF0F0F0F0u, wa1.y & 0xF0F0F0F0u, wb1.y & 0xF0F0F0F0u, q0.y, q0.w);
-                    mma_u8s8(cl0, wa0.z & 0x0F0F0F0Fu, wb0.z & 0x0F0F0F0Fu, wa0.w & 0x0F0F0F0Fu, wb0.w & 0x0F0F0F0Fu, p1.x, p1.z);
-                    mma_u8s8(cl1, wa1.z & 0x0F0F0F0Fu, wb1.z & 0x0F0F0F0Fu, wa1.w & 0x0F0F0F0Fu, wb1.w & 0x0F0F0F0Fu, q1.x, q1.z);
-                    mma_u8s8(ch0, wa0.z & 0xF0F0F0F0u, wb0.z & 0xF0F0F0F0u, wa0.w & 0xF0F0F0F0u, wb0.w & 0xF0F0F0F0u, p1.y, p1.w);
-                    mma_u8s8(ch1, wa1.z & 0xF0F0F0F0u, wb1.z & 0xF0F0F0F0u, wa1.w & 0xF0F0F0F0u, wb1.w & 0xF0F0F0F0u, q1.y, q1.w);
+                    mma_u8s8(cl0, wa0.x & LO, wb0.x & LO, wa0.y & LO, wb0.y & LO, p0.x, p0.y);
+                    mma_u8s8(cl1, wa1.x & LO, wb1.x & LO, wa1.y & LO, wb1.y & LO, q0.x, q0.y);
+                    mma_u8s8_z(ch0, wa0.x & HI, wb0.x & HI, wa0.y & HI, wb0.y & HI, p0.z, p0.w);
+                    mma_u8s8_z(ch1, wa1.x & HI, wb1.x & HI, wa1.y & HI, wb1.y & HI, q0.z, q0.w);
+                    mma_u8s8(cl0, wa0.z & LO, wb0.z & LO, wa0.w & LO, wb0.w & LO, p1.x, p1.y);
+                    mma_u8s8(cl1, wa1.z & LO, wb1.z & LO, wa1.w & LO, wb1.w & LO, q1.x, q1.y);
+                    mma_u8s8(ch0, wa0.z & HI, wb0.z & HI, wa0.w & HI, wb0.w & HI, p1.z, p1.w);
+                    mma_u8s8(ch1, wa1.z & HI, wb1.z & HI, wa1.w & HI, wb1.w & HI, q1.z, q1.w);
 #endif
                     const int d00 = (cl0[0] << 4) + ch0[0], d01 = (cl0[1] << 4) + ch0[1];      // 16 x D, exact
                     const int d02 = (cl0[2] << 4) + ch0[2], d03 = (cl0[3] << 4) + ch0[3];
                     const int d10 = (cl1[0] << 4) + ch1[0], d11 = (cl1[1] << 4) + ch1[1];
                     const int d12 = (cl1[2] << 4) + ch1[2], d13 = (cl1[3] << 4) + ch1[3];
-                    // ascending group order within the warp: the earlier group first
-                    facc[mb][0] = fmaf(s_lo1, (float)d10, fmaf(s_lo0, (float)d00, facc[mb][0]));
-                    facc[mb][1] = fmaf(s_lo1, (float)d11, fmaf(s_lo0, (float)d01, facc[mb][1]));
-                    facc[mb][2] = fmaf(s_hi1, (float)d12, fmaf(s_hi0, (float)d02, facc[mb][2]));
-                    facc[mb][3] = fmaf(s_hi1, (float)d13, fmaf(s_hi0, (float)d03, facc[mb][3]));
+                    if (SHARE) {
+                        facc[0][mb][0] = fmaf(s_lo0, (float)d00, facc[0][mb][0]);
+                        facc[0][mb][1] = fmaf(s_lo0, (float)d01, facc[0][mb][1]);
+                        facc[0][mb][2] = fmaf(s_hi0, (float)d02, facc[0][mb][2]);
+                        facc[0][mb][3] = fmaf(s_hi0, (float)d03, facc[0][mb][3]);
+                        facc[NF - 1][mb][0] = fmaf(s_lo1, (float)d10, facc[NF - 1][mb][0]);
+                        facc[NF - 1][mb][1] = fmaf(s_lo1, (float)d11, facc[NF - 1][mb][1]);
+                        facc[NF - 1][mb][2] = fmaf(s_hi1, (float)d12, facc[NF - 1][mb][2]);
+                        facc[NF - 1][mb][3] = fmaf(s_hi1, (float)d13, facc[NF - 1][mb][3]);
+                    } else {
+                        // ascending group order within the warp: the earlier group first
+                        facc[0][mb][0] = fmaf(s_lo1, (float)d10, fmaf(s_lo0, (float)d00, facc[0][mb][0]));
+                        facc[0][mb][1] = fmaf(s_lo1, (float)d11, fmaf(s_lo0, (float)d01, facc[0][mb][1]));
+                        facc[0][mb][2] = fmaf(s_hi1, (float)d12, fmaf(s_hi0, (float)d02, facc[0][mb][2]));
+                        facc[0][mb][3] = fmaf(s_hi1, (float)d13, fmaf(s_hi0, (float)d03, facc[0][mb][3]));
+                    }
                     if (DEBUG) {
                         const int m0 = 8 * mb + 2 * j;
-                        const size_t n_lo = (size_t)strip * R + row, n_hi = n_lo + 8;
+                        const size_t n0 = (size_t)strip * R + row, n1 = SHARE ? n0 + 16 : n0;
                         if (g0 < G) {
                             if (m0 < a.M) {
-                                a.debug_partials[((size_t)m0 * G + g0) * a.N + n_lo] = d00 >> 4;
-                                a.debug_partials[((size_t)m0 * G + g0) * a.N + n_hi] = d02 >> 4;
+                                a.debug_partials[((size_t)m0 * G + g0) * a.N + n0] = d00 >> 4;
+                                a.debug_partials[((size_t)m0 * G + g0) * a.N + n0 + 8] = d02 >> 4;
                             }
                             if (m0 + 1 < a.M) {
-                                a.debug_partials[((size_t)(m0 + 1) * G + g0) * a.N + n_lo] = d01 >> 4;
-                                a.debug_partials[((size_t)(m0 + 1) * G + g0) * a.N + n_hi] = d03 >> 4;
+                                a.debug_partials[((size_t)(m0 + 1) * G + g0) * a.N + n0] = d01 >> 4;
+                                a.debug_partials[((size_t)(m0 + 1) * G + g0) * a.N + n0 + 8] = d03 >> 4;
                             }
                         }
                         if (g1 < G) {
                             if (m0 < a.M) {
-                                a.debug_partials[((size_t)m0 * G + g1) * a.N + n_lo] = d10 >> 4;
-                                a.debug_partials[((size_t)m0 * G + g1) * a.N + n_hi] = d12 >> 4;
+                                a.debug_partials[((size_t)m0 * G + g1) * a.N + n1] = d10 >> 4;
+                                a.debug_partials[((size_t)m0 * G + g1) * a.N + n1 + 8] = d12 >> 4;
                             }
                             if (m0 + 1 < a.M) {
-                                a.debug_partials[((size_t)(m0 + 1) * G + g1) * a.N + n_lo] = d11 >> 4;
-                                a.debug_partials[((size_t)(m0 + 1) * G + g1) * a.N + n_hi] = d13 >> 4;
+                                a.debug_partials[((size_t)(m0 + 1) * G + g1) * a.N + n1] = d11 >> 4;
+                                a.debug_partials[((size_t)(m0 + 1) * G + g1) * a.N + n1 + 8] = d13 >> 4;
                             }
                         }
                     }
@@ -467,9 +509,13 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
             for (int item = 0; item < ITEMS; ++item) {
                 const int rb = item / MB, mb = item % MB;
                 float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                // the warps that hold this row block, in warp order: deterministic
+                constexpr bool SHARE = RBLK >= 2;
+                constexpr int WPG = SHARE ? RBLK / 2 : 1, NF = SHARE ? 2 : 1;
 #pragma unroll
-                for (int gi = 0; gi < ST_CONSUMER_WARPS / RBLK; ++gi) {     // the warps of this row block, in warp order: deterministic
-                    const float4 v = ptx::lds128f(part_lane + ((gi * RBLK + rb) * MB + mb) * 512);
+                for (int gi = 0; gi < ST_CONSUMER_WARPS / WPG; ++gi) {
+                    const int w = gi * WPG + (SHARE ? rb / 2 : 0), f = SHARE ? rb % 2 : 0;
+                    const float4 v = ptx::lds128f(part_lane + ((w * NF + f) * MB + mb) * 512);
                     acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
                 }
                 if (!has_start) {                                  // the strip's earlier groups are the previous CTA's

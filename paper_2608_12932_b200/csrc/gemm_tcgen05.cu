@@ -356,11 +356,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                 ptx::tc_fence_after_sync();
                 const uint32_t a_addr = a_lane + sa_ * A_COLS;
                 auto put = [&](const uint4& w, int j) {                  // 16 packed bytes = k 32j .. 32j+31
+                    // words 0..3 of a chunk hold the runs of four k (a0, a2), (a1, a3), (a4, a6), (a5, a7) in their
+                    // (low, high) nibbles: columns in k order are lo(x), lo(y), hi(x), hi(y), lo(z), lo(w), hi(z), hi(w)
                     ptx::tmem_st_32x8(a_addr + 8 * j,
-                                      sub_zero4(w.x & 0x0F0F0F0Fu, kz), sub_zero4((w.x >> 4) & 0x0F0F0F0Fu, kz),
-                                      sub_zero4(w.y & 0x0F0F0F0Fu, kz), sub_zero4((w.y >> 4) & 0x0F0F0F0Fu, kz),
-                                      sub_zero4(w.z & 0x0F0F0F0Fu, kz), sub_zero4((w.z >> 4) & 0x0F0F0F0Fu, kz),
-                                      sub_zero4(w.w & 0x0F0F0F0Fu, kz), sub_zero4((w.w >> 4) & 0x0F0F0F0Fu, kz));
+                                      sub_zero4(w.x & 0x0F0F0F0Fu, kz), sub_zero4(w.y & 0x0F0F0F0Fu, kz),
+                                      sub_zero4((w.x >> 4) & 0x0F0F0F0Fu, kz), sub_zero4((w.y >> 4) & 0x0F0F0F0Fu, kz),
+                                      sub_zero4(w.z & 0x0F0F0F0Fu, kz), sub_zero4(w.w & 0x0F0F0F0Fu, kz),
+                                      sub_zero4((w.z >> 4) & 0x0F0F0F0Fu, kz), sub_zero4((w.w >> 4) & 0x0F0F0F0Fu, kz));
                 };
                 put(w0, 0);
                 put(w1, 1);

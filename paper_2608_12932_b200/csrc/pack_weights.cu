@@ -15,11 +15,12 @@ pack_weights_kernel(const uint8_t* __restrict__ qw, const uint16_t* __restrict__
     const int ntile = blockIdx.x / G, g = blockIdx.x % G;
     uint8_t* blob = packed + (size_t)blockIdx.x * BLOB_BYTES;
     uint32_t* words = reinterpret_cast<uint32_t*>(blob);
-    // 2048 words: word w = row r (w/16), word-in-row kk (w%16) <- 8 consecutive codes
+    // 2048 words: word w = row r (w/16), word-in-row kk (w%16) <- four codes in its low nibbles, four in its high ones
     for (int w = threadIdx.x; w < TILE_N * 16; w += PACK_THREADS) {
         int r = w >> 4, kk = w & 15;
-        const uint2 c = *reinterpret_cast<const uint2*>(qw + (size_t)(ntile * TILE_N + r) * K + g * GROUP + kk * 8);
-        words[r * 16 + blob_chunk_pos(r, kk >> 2) * 4 + (kk & 3)] = (c.x & 0x0F0F0F0Fu) | ((c.y & 0x0F0F0F0Fu) << 4);
+        const uint8_t* src = qw + (size_t)(ntile * TILE_N + r) * K + g * GROUP + blob_word_k(kk);
+        const uint32_t lo = *reinterpret_cast<const uint32_t*>(src), hi = *reinterpret_cast<const uint32_t*>(src + 8);
+        words[r * 16 + blob_chunk_pos(r, kk >> 2) * 4 + (kk & 3)] = (lo & 0x0F0F0F0Fu) | ((hi & 0x0F0F0F0Fu) << 4);
     }
     if (threadIdx.x < TILE_N) {
         int r = threadIdx.x;
@@ -43,8 +44,9 @@ unpack_weights_kernel(const uint8_t* __restrict__ packed, int N, int K, uint8_t*
         for (int w = threadIdx.x; w < TILE_N * 16; w += PACK_THREADS) {
             int r = w >> 4, kk = w & 15;
             uint32_t v = words[r * 16 + blob_chunk_pos(r, kk >> 2) * 4 + (kk & 3)];
-            uint2 c = make_uint2(v & 0x0F0F0F0Fu, (v >> 4) & 0x0F0F0F0Fu);
-            *reinterpret_cast<uint2*>(qw + (size_t)(ntile * TILE_N + r) * K + g * GROUP + kk * 8) = c;
+            uint8_t* dst = qw + (size_t)(ntile * TILE_N + r) * K + g * GROUP + blob_word_k(kk);
+            *reinterpret_cast<uint32_t*>(dst) = v & 0x0F0F0F0Fu;
+            *reinterpret_cast<uint32_t*>(dst + 8) = (v >> 4) & 0x0F0F0F0Fu;
         }
     }
     if (threadIdx.x < TILE_N) {

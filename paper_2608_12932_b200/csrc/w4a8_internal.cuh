@@ -11,10 +11,14 @@ namespace w4a8 {
 // ---- packed weight layout -----------------------------------------------------------------
 // The [N,K] layer is cut into blobs of 128 output channels x one group of 128 k.  Blob
 // (ntile, g) sits at byte offset (ntile * G + g) * BLOB_BYTES and holds
-//   [0, 8192)     128 rows x 64 B of nibbles.  Row r, 32-bit word kk (0..15) covers
-//                 k0 = g*128 + 8*kk: byte b of the word has code[k0+b] in its low nibble and
-//                 code[k0+4+b] in its high nibble, so  w & 0x0F0F0F0F  and  (w>>4) & 0x0F0F0F0F
-//                 are four consecutive-k bytes each, and a 16-byte chunk unpacks to 32 consecutive k.
+//   [0, 8192)     128 rows x 64 B of nibbles.  Row r, 32-bit word kk (0..15) belongs to the 16-byte chunk
+//                 kk / 4, which covers 32 consecutive k.  Call the chunk's k range eight runs of four,
+//                 a0..a7.  Word q = kk % 4 of the chunk has, byte by byte, run a(4 (q / 2) + q % 2) in its
+//                 low nibbles and the run two further on in its high nibbles: words 0..3 hold
+//                 (a0, a2), (a1, a3), (a4, a6), (a5, a7).   w & 0x0F0F0F0F  and  (w >> 4) & 0x0F0F0F0F
+//                 are four consecutive-k bytes each, and the low nibbles of two neighbouring words go
+//                 with two neighbouring 4-byte words of an activation row (so do the high ones): a
+//                 warp-level MMA takes its two activation registers as they were loaded (blob_word_k).
 //                 The four 16-byte chunks of a row are stored XOR-swizzled: chunk p of row r sits at
 //                 position p ^ ((r >> 1) & 3) of the row (blob_chunk_pos).  A thread-per-row reader
 //                 (16-byte loads at a 64-byte stride) then takes its four chunks without shared-memory
@@ -25,6 +29,8 @@ namespace w4a8 {
 // A blob is exactly the algorithmic 4.15625 bits per weight: no padding.
 constexpr int TILE_N = 128;
 __host__ __device__ constexpr int blob_chunk_pos(int r, int p) { return p ^ ((r >> 1) & 3); }
+// first k (inside the group) of the four codes in the low nibbles of word kk of a row; the high nibbles start 8 later
+__host__ __device__ constexpr int blob_word_k(int kk) { return 32 * (kk >> 2) + 16 * ((kk & 3) >> 1) + 4 * (kk & 1); }
 constexpr int GROUP = 128;
 constexpr int BLOB_NIBBLE_BYTES = TILE_N * GROUP / 2;        // 8192
 constexpr int BLOB_SCALE_OFF = BLOB_NIBBLE_BYTES;             // 8192
