@@ -57,8 +57,10 @@ typedef enum {
     W4A8_PATH_TCGEN05 = 2,   /* TMA + tcgen05.mma kind::i8 + TMEM kernel (any M)             */
     W4A8_PATH_SPLITK_WORKSPACE = 3, /* split-K kernel that reduces its slices through the global
                                 workspace (M <= 64); what w4a8_gemm_static_scratch runs        */
-    W4A8_PATH_STRIP = 4      /* weight-streaming kernel without a K split: one persistent CTA per SM,
+    W4A8_PATH_STRIP = 4,     /* weight-streaming kernel without a K split: one persistent CTA per SM,
                                 strips of 16..128 channels over the whole K range dealt out evenly
+XX = 5     /* weight-streaming kernel on tcgen05: one persistent CTA per SM, the tiles x
+                                groups blobs dealt out evenly, weights unpacked into tensor memory
                                 (M <= 16)                                                       */
 } w4a8_path;
 

@@ -58,10 +58,12 @@ bool small_m_prefers_tcgen05(int M, int N, int K, int sms) {
 
 namespace {
 
-// Where w4a8_gemm takes the strip kernel: where it is measured faster than the cluster split-K kernel on B200 so far,
-// i.e. up to 8 tokens on layers with fewer 128-channel tiles than SMs.
+// Where w4a8_gemm takes the strip kernel: up to 8 tokens always; from 9 to 16 tokens (two token blocks per warp:
+// the activation tiles then crowd the ring of a narrow strip) only on layers wide enough for strips of 32 rows,
+// where it is measured faster than the cluster split-K kernel on B200.
 bool auto_takes_strip(int M, int N, int K) {
-    return strip_supported(M, N, K) && M <= 8 && N / TILE_N < device_sm_count();
+    if (!strip_supported(M, N, K)) return false;
+    return M <= 8 || N / 32 >= (device_sm_count() * 5) / 4;
 }
 
 size_t slices_bytes(int M, int N, int K) {

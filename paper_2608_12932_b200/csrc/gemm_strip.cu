@@ -462,8 +462,9 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
         // Hand-over words: a float in the low half, the tag 1 in the high half, written and read as one 64-bit
         // word each (no flag, no fence: a word says for itself that it has been written); a lane's four sums of an
         // item are two 16-byte pairs, pair h of item i at ulonglong2 index (2 i + h) * 32 + lane of the CTA's slot.
-        ulonglong2* mine = reinterpret_cast<ulonglong2*>(reinterpret_cast<uint8_t*>(a.slots) + (size_t)blockIdx.x * STRIP_SLOT_BYTES);
-        ulonglong2* theirs = reinterpret_cast<ulonglong2*>(reinterpret_cast<uint8_t*>(a.slots) + (size_t)(blockIdx.x + 1) * STRIP_SLOT_BYTES);
+        constexpr size_t SLOT = (size_t)R * MP * 8;               // a CTA's slot: one 64-bit word per sum of a strip
+        ulonglong2* mine = reinterpret_cast<ulonglong2*>(reinterpret_cast<uint8_t*>(a.slots) + (size_t)blockIdx.x * SLOT);
+        ulonglong2* theirs = reinterpret_cast<ulonglong2*>(reinterpret_cast<uint8_t*>(a.slots) + (size_t)(blockIdx.x + 1) * SLOT);
         constexpr unsigned long long TAG = 1ull << 32;
         for (int q = 0; q < nseg && ok; ++q) {
             const int strip = first_strip + q;
@@ -639,24 +640,32 @@ bool strip_supported(int M, int N, int K) {
     return M >= 1 && M <= STRIP_MAX_M && (K / GROUP) * mp <= ST_MAX_ASUM_WORDS && N >= 16;
 }
 
-// Strip width and CTA count for a problem.  The widest strip that still gives about one strip per SM:
-// wide strips share an activation tile between more rows (less traffic from L2 into shared memory); a
-// narrow one is needed where a layer has fewer 128-channel tiles than the device has SMs.  The grid never
-// exceeds the number of strips, so that a strip is shared by at most two CTAs.
+// Strip width and CTA count for a problem (measured on B200, sweep of widths 16..128 and 148..296 CTAs on the
+// four layer shapes of an 8B-class decoder, 4 to 16 tokens): the widest strip that still gives about 1.25 strips
+// per SM, and up to two CTAs per SM - the second CTA's warps multiply while the first one's wait for data, which is
+// worth more than a whole SM's shared memory held free for the next launch; the next launch's CTAs still start
+// (and prefetch) as soon as the first CTAs of this one leave.  Wide strips share an activation tile between more
+// rows (less traffic from L2 into shared memory); 16-row strips are left to up to 8 tokens, where their 16
+// activation tiles per stage still leave room for a ring.  The grid never exceeds the number of strips, so that a
+// strip is shared by at most two CTAs.
 void strip_plan(int M, int N, int K, int* strip_rows, int* ctas) {
     (void)K;
     const int sms = device_sm_count();
-    const int limit = sms < STRIP_MAX_CTAS ? sms : STRIP_MAX_CTAS;
-    // 16-row strips carry 16 groups' activation tiles per stage: with two token blocks that leaves no room for a ring
     const int r_min = M <= 8 ? 16 : 32;
     int R = 128;
-    while (R > r_min && N / R < (limit * 17) / 20) R /= 2;      // at least 0.85 strips per SM
+    while (R > r_min && N / R < (sms * 5) / 4) R /= 2;
 #ifdef W4A8_TUNING
     if (const char* e = getenv("W4A8_STRIP_R")) {
         const int v = atoi(e);
         if (v == 16 || v == 32 || v == 64 || v == 128) R = v;
     }
 #endif
+    int limit = 2 * sms;
+#ifdef W4A8_TUNING
+    if (const char* e = getenv("W4A8_STRIP_CTAS")) { const int v = atoi(e); if (v >= 1) limit = v; }
+#endif
+    const int slot_limit = (STRIP_MAX_CTAS * STRIP_SLOT_BYTES) / (R * (M <= 8 ? 8 : 16) * 8);    // hand-over slots in the workspace
+    if (limit > slot_limit) limit = slot_limit;
     int c = N / R;
     if (c > limit) c = limit;
     if (strip_rows) *strip_rows = R;

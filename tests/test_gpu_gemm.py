@@ -100,14 +100,15 @@ def test_strip_token_counts(mid_case, M):
 
 # layer shapes chosen for the strip widths the planner picks on 148 SMs and for how the strips fall on the CTAs
 STRIP_SHAPES = [
-    (512, 128, 16),       # 8 strips of 16 channels, 8 CTAs with one strip each, one stage (half a ring) per strip
-    (1280, 2432, 16),     # 152 strips of 16 on 148 CTAs: nearly every strip is shared by two CTAs; 10 groups in stages of 8
-    (1024, 4736, 32),     # 148 strips of 32: exactly one per CTA
-    (3072, 6144, 32),     # 192 strips of 32, 24 groups: ranges of 1.3 strips, ring re-used
-    (640, 12288, 64),     # 192 strips of 64, 5 groups in stages of 2 (a ragged last stage)
-    (896, 18944, 128),    # 148 strips of 128
-    (384, 24576, 128),    # 192 strips of 128, 3 groups: ranges shorter than the ring
-    (4096, 37888, 128),   # 296 strips of 128: two whole strips per CTA, no hand-over
+    (512, 128, 16),       # 8 strips of 16 channels, 8 CTAs with one strip each, one ragged stage per strip
+    (1280, 2432, 16),     # 152 strips of 16, one per CTA; 10 groups in stages of 16
+    (1024, 4864, 16),     # 304 strips of 16 on 296 CTAs: nearly every strip is shared by two CTAs
+    (3072, 6144, 32),     # 192 strips of 32, 24 groups in stages of 8
+    (640, 12288, 64),     # 192 strips of 64, 5 groups in stages of 4 (a ragged last stage)
+    (896, 37888, 128),    # 296 strips of 128: exactly one per CTA
+    (384, 24576, 128),    # 192 strips of 128, 3 groups in stages of 2
+    (1024, 49152, 128),   # 384 strips of 128 on 296 CTAs: ranges of 1.3 strips, hand-over
+    (4096, 12288, 64),    # 192 strips of 64, 32 groups: the ring re-used
 ]
 
 
@@ -122,7 +123,7 @@ def test_strip_widths_and_hand_over(K, N, rows):
     for M in (8, 16, 5):
         plan = B.w4a8_plan(M, N, K)
         if plan["family"] == B.PATH_STRIP:
-            assert plan["k_slices"] == 1 and plan["ctas"] <= min(sms, N // plan["strip_rows"])
+            assert plan["k_slices"] == 1 and plan["ctas"] <= min(2 * sms, N // plan["strip_rows"])
             if sms == 148:
                 assert plan["strip_rows"] == (rows if M <= 8 else max(rows, 32)), plan
         y1, _, _ = check_case(case, layer, M, "strip", debug=(K * N <= 1 << 26))
@@ -485,7 +486,7 @@ def test_plan_matches_the_device():
     p = B.w4a8_plan(64, 4096, 12288)                  # down projection, 32 tiles, 96 groups
     assert p["family"] == B.PATH_TCGEN05 and p["k_slices"] > 1 and p["ctas"] <= sms
     p = B.w4a8_plan(8, 6144, 4096)
-    assert (p["family"] == B.PATH_STRIP and p["ctas"] == min(sms, 6144 // p["strip_rows"]) and p["k_slices"] == 1) or \
+    assert (p["family"] == B.PATH_STRIP and p["ctas"] == min(2 * sms, 6144 // p["strip_rows"]) and p["k_slices"] == 1) or \
         (p["family"] == B.PATH_SPLITK and p["ctas"] == 48 * p["k_slices"])
     p = B.w4a8_plan(40, 6144, 4096)
     assert (p["family"] == B.PATH_SPLITK and p["ctas"] == 48 * p["k_slices"]) or p["family"] == B.PATH_TCGEN05

@@ -73,14 +73,14 @@ def test_plan_query_invariants():
             if M > 64:
                 assert p["family"] == B.PATH_TCGEN05
             if p["family"] == B.PATH_STRIP:
-                # one strip per CTA at least, so that a strip is shared by at most two CTAs; never a K split
+                # at most two CTAs per SM, one strip per CTA at least (a strip is shared by at most two CTAs); never a K split
                 R = p["strip_rows"]
                 assert R in (16, 32, 64, 128) and p["k_slices"] == 1 and p["tile_m"] == (8 if M <= 8 else 16)
-                assert 1 <= p["ctas"] <= min(sms, N // R)
+                assert 1 <= p["ctas"] <= min(2 * sms, N // R)
                 assert p["balanced"] == int((N // R) % p["ctas"] != 0)
-                # the widest strip that keeps about 0.85 strips per SM
-                assert R == 128 or N // (2 * R) < (sms * 17) // 20
-                assert R == (16 if M <= 8 else 32) or N // R >= (sms * 17) // 20
+                # the widest strip that keeps about 1.25 strips per SM
+                assert R == 128 or N // (2 * R) < (sms * 5) // 4
+                assert R == (16 if M <= 8 else 32) or N // R >= (sms * 5) // 4
             elif p["family"] == B.PATH_SPLITK:
                 assert p["strip_rows"] == 0
                 assert p["tile_m"] in (8, 16, 32, 64) and p["tile_m"] >= min(M, 64)
