@@ -642,7 +642,7 @@ bool strip_supported(int M, int N, int K) {
 
 // Strip width and CTA count for a problem (measured on B200, sweep of widths 16..128 and 148..296 CTAs on the
 // four layer shapes of an 8B-class decoder, 4 to 16 tokens): the widest strip that still gives about 1.25 strips
-// per SM, and up to two CTAs per SM - the second CTA's warps multiply while the first one's wait for data, which is
+// per SM (one step narrower if a wide strip would leave SMs with a single CTA), and up to two CTAs per SM - the second CTA's warps multiply while the first one's wait for data, which is
 // worth more than a whole SM's shared memory held free for the next launch; the next launch's CTAs still start
 // (and prefetch) as soon as the first CTAs of this one leave.  Wide strips share an activation tile between more
 // rows (less traffic from L2 into shared memory); 16-row strips are left to up to 8 tokens, where their 16
@@ -651,9 +651,13 @@ bool strip_supported(int M, int N, int K) {
 void strip_plan(int M, int N, int K, int* strip_rows, int* ctas) {
     (void)K;
     const int sms = device_sm_count();
-    const int r_min = M <= 8 ? 16 : 32;
     int R = 128;
-    while (R > r_min && N / R < (sms * 5) / 4) R /= 2;
+    if (M <= 8) {
+        while (R > 16 && N / R < (sms * 5) / 4) R /= 2;
+        if (R > 32 && N / R < 2 * sms) R /= 2;               // wide strips: enough of them for two CTAs on every SM
+    } else {
+        R = 32;                                              // two token blocks: 32-row strips measured best (wider: fewer CTAs or more
+    }                                                        // hand-over; narrower: the activation tiles crowd the ring)
 #ifdef W4A8_TUNING
     if (const char* e = getenv("W4A8_STRIP_R")) {
         const int v = atoi(e);

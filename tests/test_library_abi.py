@@ -78,9 +78,12 @@ def test_plan_query_invariants():
                 assert R in (16, 32, 64, 128) and p["k_slices"] == 1 and p["tile_m"] == (8 if M <= 8 else 16)
                 assert 1 <= p["ctas"] <= min(2 * sms, N // R)
                 assert p["balanced"] == int((N // R) % p["ctas"] != 0)
-                # the widest strip that keeps about 1.25 strips per SM
-                assert R == 128 or N // (2 * R) < (sms * 5) // 4
-                assert R == (16 if M <= 8 else 32) or N // R >= (sms * 5) // 4
+                if M > 8:
+                    assert R == 32
+                else:
+                    # the widest strip that keeps about 1.25 strips per SM, one step narrower if that leaves fewer than two per SM
+                    assert R == 16 or N // R >= (sms * 5) // 4
+                    assert R >= 64 or N // (2 * R) < (sms * 5) // 4 or (R == 32 and N // 64 < 2 * sms)
             elif p["family"] == B.PATH_SPLITK:
                 assert p["strip_rows"] == 0
                 assert p["tile_m"] in (8, 16, 32, 64) and p["tile_m"] >= min(M, 64)
