@@ -242,6 +242,17 @@ w4a8_status w4a8_gemm_static_scratch(const int8_t* qa, const uint16_t* sa, const
 w4a8_status w4a8_static_scratch_status(void* stream);
 
 /*
+ * Self-test of the kernels' give-up path (no counterpart in the paper).  Runs the workspace split-K kernel on the
+ * given problem (M <= 64) in a form in which every CTA leaves one of its weight copies out and waits for at most
+ * 200 microseconds: the wait expires, the CTA records W4A8_ERR_TIMEOUT in the workspace status word, waits (again
+ * bounded) for its copies in flight and the kernel returns normally.  y_bf16 is written but invalid.  Afterwards
+ * w4a8_check_status returns W4A8_ERR_TIMEOUT once and the workspace is usable as before.  Nothing faults or hangs.
+ */
+w4a8_status w4a8_selftest_wait_timeout(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed_w,
+                                       void* y_bf16, int M, int N, int K, int group, void* workspace,
+                                       size_t workspace_bytes, void* stream);
+
+/*
  * Reads back the workspace status word: synchronises `stream`, returns W4A8_OK or
  * W4A8_ERR_TIMEOUT (a kernel gave up on a bounded wait; its output is then invalid), and
  * clears the word.  Host-synchronising: for tests and debugging, not for the hot path.

@@ -21,7 +21,7 @@ WORKSPACE_ZEROED_BYTES = 4096 + 192 * 16384
 EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w4a8_workspace_init",
            "w4a8_pack_weights", "w4a8_unpack_weights", "w4a8_quantize_act", "w4a8_gemm", "w4a8_gemm_path",
            "w4a8_linear", "w4a8_linear_host", "w4a8_gemm_static_scratch", "w4a8_check_status", "w4a8_plan",
-           "w4a8_gemm_per_channel", "w4a8_static_scratch_status")
+           "w4a8_gemm_per_channel", "w4a8_static_scratch_status", "w4a8_selftest_wait_timeout")
 
 _lib = None
 
@@ -71,6 +71,8 @@ def lib():
         L.w4a8_gemm_static_scratch.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp]
         L.w4a8_check_status.restype = ci
         L.w4a8_check_status.argtypes = [vp, vp]
+        L.w4a8_selftest_wait_timeout.restype = ci
+        L.w4a8_selftest_wait_timeout.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp]
         L.w4a8_static_scratch_status.restype = ci
         L.w4a8_static_scratch_status.argtypes = [vp]
         _lib = L
@@ -254,6 +256,15 @@ def w4a8_gemm_static_scratch(qa, sa, asum, packed_w, N, group=GROUP, out=None, s
 
 def w4a8_check_status(workspace, stream=None):
     _check(lib().w4a8_check_status(_ptr(workspace), _stream(stream)), "w4a8_check_status")
+
+
+def w4a8_selftest_wait_timeout(qa, sa, asum, packed_w, N, workspace, group=GROUP, stream=None):
+    """Runs the split-K kernel with one weight copy withheld per CTA and a 200 us wait limit (see w4a8.h); returns y (invalid)."""
+    M, K = qa.shape
+    out = torch.empty((M, N), dtype=torch.bfloat16, device=qa.device)
+    _check(lib().w4a8_selftest_wait_timeout(_ptr(qa), _ptr(sa), _ptr(asum), _ptr(packed_w), _ptr(out), M, N, K, group,
+                                            _ptr(workspace), workspace.numel(), _stream(stream)), "w4a8_selftest_wait_timeout")
+    return out
 
 
 def w4a8_static_scratch_status(stream=None):

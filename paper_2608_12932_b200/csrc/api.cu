@@ -292,6 +292,22 @@ w4a8_status w4a8_check_status(void* workspace, void* stream) {
     return word == W4A8_ERR_TIMEOUT ? W4A8_ERR_TIMEOUT : W4A8_ERR_CUDA;
 }
 
+w4a8_status w4a8_selftest_wait_timeout(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed_w,
+                                       void* y_bf16, int M, int N, int K, int group, void* workspace,
+                                       size_t workspace_bytes, void* stream) {
+    if (!shape_ok(N, K, group) || M <= 0 || M > SPLITK_MAX_M) return W4A8_ERR_SHAPE;
+    if (!qa || !sa || !asum || !packed_w || !y_bf16 || !workspace) return W4A8_ERR_NULL;
+    if (!aligned(qa, 16) || !aligned(sa, 2) || !aligned(asum, 4) || !aligned(packed_w, 128) || !aligned(y_bf16, 2) ||
+        !aligned(workspace, 256))
+        return W4A8_ERR_ALIGN;
+    if (workspace_bytes < w4a8_workspace_bytes(M, N, K, group)) return W4A8_ERR_WORKSPACE;
+    w4a8_status a = arch_check();
+    if (a != W4A8_OK) return a;
+    return launch_gemm_splitk(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace,
+                              reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + WS_SHARED_OFF), withhold_marker(),
+                              static_cast<cudaStream_t>(stream)) == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
 w4a8_status w4a8_static_scratch_status(void* stream) {
     void* scratch = static_scratch_address();        // looks the array's device address up; allocates nothing
     if (!scratch) return W4A8_ERR_CUDA;

@@ -62,6 +62,7 @@ inline size_t handover_bytes(int M, int N, int /*K*/) {
 constexpr int SPLITK_MAX_M = 64;          // tokens the streaming kernel handles (8 blocks of 8)
 constexpr int SPLITK_MAX_GROUPS = 8;      // groups one CTA keeps in shared memory at once
 int splitk_num_slices(int M, int N, int K);
+int32_t* withhold_marker();
 
 cudaError_t make_qa_tensor_map(CUtensorMap* out, const int8_t* qa, int M, int K, int box_rows);
 cudaError_t make_y_tensor_map(CUtensorMap* out, void* y, int M, int N);

@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import cfast
 from oracle import w4a8_oracle as onp
 from paper_2608_12932_b200 import binding as B
 from paper_2608_12932_b200 import workload as wl
@@ -37,6 +38,12 @@ def test_static_scratch_matches_workspace_entry_point_twice():
         assert np.array_equal(got, want), f"call {call}: same kernel, same inputs, different bits"
         ok, ratio = onp.within_tolerance(got, onp.bf16_bits_to_f64(auto))
         assert ok, f"call {call} against w4a8_gemm: worst |err|/bound = {ratio}"
+        # and against the CPU oracle, which shares nothing with either entry point
+        ref = cfast.w4a8_linear(case["x"][:M], case["qw"], case["sw"], case["z"], case["group"])
+        ok, ratio = onp.within_tolerance(got, ref["ref"])
+        assert ok, f"call {call} against the oracle: worst |err|/bound = {ratio}"
+        # the status word of this path lives in the fixed array: readable without a workspace pointer
+        B.w4a8_static_scratch_status()
 
 
 def test_static_scratch_second_call_same_shape_and_limits():
