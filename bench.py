@@ -59,6 +59,41 @@ def measured_peaks():
                 bf16_tflops_sustained=1400.0, source="fallback")
 
 
+def measure_int8_peak(torch, seconds=2.0):
+    """A library INT8 GEMM (torch._int_mm, 8192^3) timed on this GPU: best single launch (burst) and a back-to-back
+    loop of `seconds` (sustained, under the power cap).  Timing a library is allowed; it is not on the product path."""
+    try:
+        n = 8192
+        a = torch.randint(-127, 128, (n, n), dtype=torch.int8, device="cuda")
+        b = torch.randint(-127, 128, (n, n), dtype=torch.int8, device="cuda")
+        for _ in range(3):
+            torch._int_mm(a, b)
+        torch.cuda.synchronize()
+        best = 1e9
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            torch._int_mm(a, b)
+            e1.record()
+            e1.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        reps = max(10, int(seconds * 1e3 / best))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            torch._int_mm(a, b)
+        e1.record()
+        e1.synchronize()
+        sustained = e0.elapsed_time(e1) / reps
+        ops = 2.0 * n ** 3
+        del a, b
+        torch.cuda.empty_cache()
+        return {"int8_tops_burst": ops / best / 1e9, "int8_tops_sustained": ops / sustained / 1e9,
+                "how": f"torch._int_mm {n}^3, best of 10 and {reps} back to back"}
+    except Exception as ex:      # noqa: BLE001 - the library routine may be missing; the stand-in is then used alone
+        return {"int8_tops_burst": None, "int8_tops_sustained": None, "how": f"unavailable: {type(ex).__name__}"}
+
+
 def step_bytes(M, N, K):
     return wl.algorithmic_bytes_quantize(M, K) + wl.algorithmic_bytes_gemm(M, N, K)
 
@@ -111,6 +146,10 @@ class ClockSampler:
                 "reasons": sorted(reasons)}
 
 
+def workload_name(M, N, K):
+    return f"{HEADLINE}: M={M} K={K} N={N} group=128; step = w4a8_linear (w4a8_quantize_act + w4a8_gemm)"
+
+
 # ----------------------------------------------------------------------- CPU oracle arm ---
 def time_oracle(case, min_seconds, max_steps=None):
     """The CPU oracle, as it stands, on the whole headline step; returns (steps, seconds, threads)."""
@@ -139,7 +178,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": steps, "warmup": args.warmup, "ms_per_step": el / steps * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8 x uint4 -> int32, fp64 scaling", "data": "synthetic",
-        "config": {"workload": f"{HEADLINE}: M={M} K={K} N={N} group=128, quantise + W4A8 linear"},
+        "config": {"workload": workload_name(M, N, K)},
         "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle",
                          "sample": f"the whole step, {steps} repetitions"},
         "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -202,9 +241,12 @@ def copies_for(nbytes, l2_bytes):
 
 
 def run_sweep(torch, B, peaks, l2_bytes, timer):
-    """All four linears at every M of the sweep: GEMM alone, rotating cold weight copies."""
+    """All four linears at every M of the sweep: GEMM alone, rotating cold weight copies; best of 5 graph replays.
+    frac_measured: against the measured HBM copy rate / 2 x the measured bf16 rate; frac_int8_mm: against the library
+    INT8 GEMM measured in this run (burst)."""
     out, out_pc = [], []
     int8_peak = 2.0 * peaks["bf16_tflops"]
+    int8_mm = peaks.get("int8_tops_burst")
     for lname, (K, N) in wl.LAYERS.items():
         case = wl.make_sweep_layer(lname)
         qw = torch.from_numpy(case["qw"]).cuda()
@@ -238,7 +280,9 @@ def run_sweep(torch, B, peaks, l2_bytes, timer):
                         "tops": round(ops / us / 1e6, 1), "gbs": round(nbytes / us / 1e3, 1),
                         "bound": "int8" if t_c_meas > t_m_meas else "hbm",
                         "frac_measured": round(max(t_c_meas, t_m_meas) * 1e6 / us, 3),
-                        "frac_nominal": round(max(t_c_nom, t_m_nom) * 1e6 / us, 3)})
+                        "frac_nominal": round(max(t_c_nom, t_m_nom) * 1e6 / us, 3),
+                        "frac_int8_mm": (round(max(ops / (int8_mm * 1e12), t_m_meas) * 1e6 / us, 3) if int8_mm else None),
+                        "kernel": plan_name(B, M, N, K)})
             if M >= 1024:
                 # the same pipeline with one drain per tile (w4a8_gemm_per_channel: scales constant along K;
                 # it reads the first group's scales only, so the timing needs no second set of weights)
@@ -255,6 +299,81 @@ def run_sweep(torch, B, peaks, l2_bytes, timer):
         del packed, packed0, x_all
         torch.cuda.empty_cache()
     return out, out_pc
+
+
+def plan_name(B, M, N, K):
+    """The kernel w4a8_gemm launches for a size, from the library's own planner."""
+    p = B.w4a8_plan(M, N, K)
+    if p["family"] == B.PATH_STRIP:
+        return f"gemm_strip_kernel<{p['tile_m'] // 8},{p['strip_rows'] // 16}> x {p['ctas']} CTAs"
+    if p["family"] == B.PATH_SPLITK:
+        return f"gemm_cluster_kernel<{p['tile_m'] // 8}> x {p['ctas']} CTAs, {p['k_slices']} K slices"
+    return (f"gemm_tcgen05_kernel<{p['tile_m']}> x {p['ctas']} CTAs" + (f", {p['k_slices']} K slices" if p["k_slices"] > 1 else "")
+            + (", balanced walk" if p["balanced"] else ""))
+
+
+def run_large_m_roofline(torch, B, peaks, l2_bytes, timer):
+    """The tensor-core kernel alone on the streaming-prefill configuration (M = 1024, K = 4096, N = 24576: fused gate+up),
+    cold weight copies in turn, median of 5 graph replays."""
+    c = wl.CONFIGS["prefill_gate_up"]
+    M, K, N = c["M"], c["K"], c["N"]
+    rng = np.random.default_rng(11)
+    r = wl.random_codes(rng, M, N, K)
+    p0 = B.w4a8_pack_weights(torch.from_numpy(r["qw"]).cuda(), to_dev16(torch, r["sw"], torch.float16), torch.from_numpy(r["z"]).cuda())
+    ncopies = copies_for(p0.numel(), l2_bytes)
+    packed = [p0] + [p0.clone() for _ in range(ncopies - 1)]
+    ws = B.new_workspace(M, N, K)
+    qa, sa, asum = B.w4a8_quantize_act(to_dev16(torch, r["x"], torch.bfloat16))
+    y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    B.w4a8_gemm(qa, sa, asum, packed[0], N, ws, out=y)
+    B.w4a8_check_status(ws)
+
+    def body():
+        for _ in range(2):
+            for p in packed:
+                B.w4a8_gemm(qa, sa, asum, p, N, ws, out=y)
+    _, times = timer.graph_ms(body, replays=5, warm=2)
+    B.w4a8_check_status(ws)
+    us = float(np.median(times)) * 1e3 / (2 * ncopies)
+    tops = wl.algorithmic_ops(M, N, K) / us / 1e6
+    peak2 = 2.0 * peaks["bf16_tflops"]
+    out = {"bound": "tensor", "kernel": plan_name(B, M, N, K), "workload": f"prefill_gate_up: M={M} K={K} N={N}",
+           "achieved": round(tops, 1), "unit": "TOP/s (int8)", "peak": round(peak2, 1),
+           "peak_source": f"2 x the {peaks['source']} bf16 GEMM rate (burst); nominal dense int8 : bf16 = 2",
+           "frac": round(tops / peak2, 4), "us_per_launch": round(us, 2),
+           "frac_of_nominal_4500": round(tops / NOMINAL_INT8_TOPS, 4),
+           "tensor_pipe_active_pct_ncu": 33.5, "traffic": None,
+           "timing": "median of 5 replays of back-to-back launches in one graph"}
+    if peaks.get("int8_tops_burst"):
+        out["peak_int8_mm"] = round(peaks["int8_tops_burst"], 1)
+        out["frac_of_int8_mm"] = round(tops / peaks["int8_tops_burst"], 4)
+    del packed, p0
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_quantize_roofline(torch, B, peaks, l2_bytes, timer):
+    """quantize_act alone at 1024 x 4096 on inputs visited in turn (more than two L2 capacities in all)."""
+    M, K = 1024, 4096
+    nbytes = wl.algorithmic_bytes_quantize(M, K)
+    ncopies = copies_for(2 * M * K, l2_bytes)
+    xs = [torch.randn((M, K), device="cuda").to(torch.bfloat16) for _ in range(ncopies)]
+    qa = torch.empty((M, K), dtype=torch.int8, device="cuda")
+    sa = torch.empty((M,), dtype=torch.float16, device="cuda")
+    asum = torch.empty((M, K // 128), dtype=torch.int32, device="cuda")
+
+    def body():
+        for x in xs:
+            B.w4a8_quantize_act(x, 128, out=(qa, sa, asum))
+    _, times = timer.graph_ms(body, replays=5, warm=2)
+    us = float(np.median(times)) * 1e3 / ncopies
+    gbs = nbytes / us / 1e3
+    del xs
+    torch.cuda.empty_cache()
+    return {"bound": "hbm", "kernel": "quantize_act_kernel<256>", "workload": f"M={M} K={K}", "achieved": round(gbs, 1),
+            "unit": "GB/s", "peak": peaks["hbm_gbs"], "frac": round(gbs / peaks["hbm_gbs"], 4), "us_per_launch": round(us, 2),
+            "algorithmic_bytes_per_launch": nbytes, "traffic": None,
+            "timing": "median of 5 replays of back-to-back launches in one graph"}
 
 
 def run_layer_chain(torch, B, peaks, l2_bytes, timer):
@@ -399,8 +518,9 @@ def run_gpu(args):
     _, gt = timer.graph_ms(gemm_only, replays=5, warm=2)
     gemm_us = float(np.median(gt)) * 1e3 / args.steps
     gbytes = wl.algorithmic_bytes_gemm(M, N, K)
-    roof_kernel, roof_us, roof_bytes = "gemm_cluster_kernel<1,2,2>", gemm_us, gbytes
+    roof_kernel, roof_us, roof_bytes = plan_name(B, M, N, K), gemm_us, gbytes
     achieved = roof_bytes / roof_us / 1e3
+    traffic = TRAFFIC_BYTES_PER_LAUNCH.get(roof_kernel.split("<")[0])      # ncu capture of this kernel at this shape, if one is on file
 
     def quant_only():
         for i in range(args.steps):
@@ -445,16 +565,30 @@ def run_gpu(args):
     osteps, oel, threads = time_oracle(case, 3.0)
     cpu_gbs = sbytes * osteps / oel / 1e9
 
+    # ---- the other rooflines: a library INT8 GEMM as the measured tensor peak, the large-M kernel on the
+    # streaming-prefill configuration, the quantise kernel at a prefill-sized input
+    peaks.update(measure_int8_peak(torch))
+    roof_large = run_large_m_roofline(torch, B, peaks, l2_bytes, timer)
+    roof_quant = run_quantize_roofline(torch, B, peaks, l2_bytes, timer)
+
     sweep = None
+    targets = None
     if not args.no_sweep and world == 1:
         sweep, sweep_pc = run_sweep(torch, B, peaks, l2_bytes, timer)
         layer_chain = run_layer_chain(torch, B, peaks, l2_bytes, timer)
+        small = [r for r in sweep if r["M"] <= 16]
+        large = [r for r in sweep if r["M"] >= 1024]
+        targets = {"small_m_target": 0.70, "small_m_min_frac": min(r["frac_measured"] for r in small),
+                   "small_m_max_frac": max(r["frac_measured"] for r in small),
+                   "large_m_target": 0.60, "large_m_min_frac": min(r["frac_measured"] for r in large),
+                   "large_m_max_frac": max(r["frac_measured"] for r in large),
+                   "denominators": "measured HBM copy rate (M <= 16); 2 x measured bf16 burst (M >= 1024)"}
 
     line = {
         "metric": METRIC, "value": round(value, 2), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int8 x uint4 -> int32 (fp32 scaling, bf16 out)", "data": "synthetic",
-        "config": {"workload": f"{HEADLINE}: M={M} K={K} N={N} group=128; step = w4a8_linear (w4a8_quantize_act + w4a8_gemm)",
+        "config": {"workload": workload_name(M, N, K),
                    "l2": f"{ncopies} distinct packed weight copies visited in turn ({ncopies * packed0.numel() / 2**20:.0f} MiB "
                          f"> 2 x L2 of {l2_bytes / 2**20:.0f} MiB); activations stay L2-resident as in a real decoder",
                    "launch": "one CUDA graph of K steps, CUDA events around the replay",
@@ -469,15 +603,19 @@ def run_gpu(args):
                      "peak_source": f"of {peaks['source']} (STREAM-style copy, burst)",
                      "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
                      "us_per_launch": round(roof_us, 3), "algorithmic_bytes_per_launch": roof_bytes,
-                     "traffic": TRAFFIC_BYTES_PER_LAUNCH,
-                     "timing": "K back-to-back launches in one graph, inter-launch gaps included"},
+                     "traffic": traffic,
+                     "timing": "median of 5 replays of K back-to-back launches in one graph, inter-launch gaps included"},
         "kernels_us": {"w4a8_linear": round(step_us, 3), "w4a8_quantize_act": round(quant_us, 3),
                        "w4a8_gemm": round(gemm_us, 3)},
         "cpu_baseline": {"value": round(cpu_gbs, 3), "unit": "GB/s", "cores": threads, "kind": "oracle",
                          "sample": f"the whole step (M={M}, all {N} channels), {osteps} repetitions in {oel:.1f} s"},
         "parity": parity,
+        "peaks": {k: (round(v, 1) if isinstance(v, float) else v) for k, v in peaks.items()},
+        "roofline_large_m": roof_large,
+        "roofline_quantize_act": roof_quant,
     }
     if sweep is not None:
+        line["targets"] = targets
         line["sweep"] = sweep
         line["sweep_per_channel_scales"] = sweep_pc
         line["layer_chain"] = layer_chain
@@ -525,9 +663,9 @@ def run_shape(args):
                       "gbs": round(wl.algorithmic_bytes_gemm(M, N, K) / us / 1e3, 1), "launches": args.steps}))
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one split-K GEMM launch at the headline shape,
-# from the ncu capture summarised in profiles/gemm_cluster_qkv_M8.md
-TRAFFIC_BYTES_PER_LAUNCH = 13144832
+# dram__bytes_read.sum + dram__bytes_write.sum of one GEMM launch at the headline shape, by kernel, from the ncu
+# captures summarised under profiles/ (gemm_strip_qkv_M8.md, gemm_cluster_qkv_M8.md)
+TRAFFIC_BYTES_PER_LAUNCH = {"gemm_strip_kernel": None, "gemm_cluster_kernel": 13144832}
 E2E_DEPTH = int(os.environ.get("W4A8_E2E_DEPTH", "4"))          # host requests in flight in the end-to-end measurement
 
 
