@@ -372,7 +372,7 @@ def run_quantize_roofline(torch, B, peaks, l2_bytes, timer):
     torch.cuda.empty_cache()
     return {"bound": "hbm", "kernel": "quantize_act_kernel<256>", "workload": f"M={M} K={K}", "achieved": round(gbs, 1),
             "unit": "GB/s", "peak": peaks["hbm_gbs"], "frac": round(gbs / peaks["hbm_gbs"], 4), "us_per_launch": round(us, 2),
-            "algorithmic_bytes_per_launch": nbytes, "traffic": None,
+            "algorithmic_bytes_per_launch": nbytes, "traffic": 8427520,
             "timing": "median of 5 replays of back-to-back launches in one graph"}
 
 
@@ -665,7 +665,7 @@ def run_shape(args):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one GEMM launch at the headline shape, by kernel, from the ncu
 # captures summarised under profiles/ (gemm_strip_qkv_M8.md, gemm_cluster_qkv_M8.md)
-TRAFFIC_BYTES_PER_LAUNCH = {"gemm_strip_kernel": None, "gemm_cluster_kernel": 13144832}
+TRAFFIC_BYTES_PER_LAUNCH = {"gemm_strip_kernel": 13148416, "gemm_cluster_kernel": 13144832}
 E2E_DEPTH = int(os.environ.get("W4A8_E2E_DEPTH", "4"))          # host requests in flight in the end-to-end measurement
 
 
