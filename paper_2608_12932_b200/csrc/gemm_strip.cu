@@ -55,20 +55,26 @@ namespace {
 // Eight consumer warps, each taking two of a stage's sixteen units (the same 16 rows of two groups): with twelve
 // warps in the CTA two CTAs per SM leave 80 registers per thread, enough to keep every per-lane offset in a
 // register.  (Sixteen thin warps at 48 registers re-derived them from the thread index in every unit: 119
-// instructions per unit, more than half of them address arithmetic.)
-constexpr int ST_CONSUMER_WARPS = 8;
+// instructions per unit, more than half of them address arithmetic.  Twelve consumer warps at 64 registers and
+// 24-unit stages, -DST_CW=12, give the same results 10 % slower: 14.4 against 12.9 us on the 4096 -> 24576 layer.)
+#ifndef ST_CW
+#define ST_CW 8
+#endif
+constexpr int ST_CONSUMER_WARPS = ST_CW;
+constexpr int ST_UNITS = 2 * ST_CONSUMER_WARPS;           // units (16 rows x one group) per stage
+constexpr int ST_NIB_BYTES = ST_UNITS * 1024;             // nibbles of a stage
 constexpr int ST_PRODUCER_WARPS = 3;
 constexpr int ST_EPILOGUE_WARP = ST_CONSUMER_WARPS + ST_PRODUCER_WARPS;
 constexpr int ST_THREADS = (ST_CONSUMER_WARPS + ST_PRODUCER_WARPS + 1) * 32;
 constexpr int ST_MAX_STAGES = 8;
-constexpr int ST_W_BYTES = 17408;                         // weight part of a stage (16 KB of nibbles + scales + zero points, padded)
+constexpr int ST_W_BYTES = ST_CW == 8 ? 17408 : 26624;                         // weight part of a stage (16 KB of nibbles + scales + zero points, padded)
 constexpr int ST_SMEM_BUDGET = 112 * 1024;                // per CTA: two launches share an SM
 constexpr int ST_MAX_ASUM_WORDS = 4096;                   // group sums of all tokens kept in shared memory
 
 struct StLayout {
     int ring_off, bar_off, asum_off, sa_off, part_off, take_off, ystage_off, misc_off, total;
 };
-__host__ __device__ constexpr int st_stage_bytes(int mb, int rblk) { return ST_W_BYTES + (16 / rblk) * 8 * mb * GROUP; }
+__host__ __device__ constexpr int st_stage_bytes(int mb, int rblk) { return ST_W_BYTES + (ST_UNITS / rblk) * 8 * mb * GROUP; }
 __host__ __device__ inline StLayout st_layout(int mb, int rblk, int stages, int G) {
     const int mp = 8 * mb;
     StLayout L;
@@ -158,18 +164,18 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
     const unsigned int trace_launch = trace_launch_s;
     if (threadIdx.x == 0) ST_STAMP(0);
 #endif
-    constexpr int R = 16 * RBLK, GS = 16 / RBLK, MP = 8 * MB;
+    constexpr int R = 16 * RBLK, GS = ST_UNITS / RBLK, MP = 8 * MB;
     constexpr int STRIPS_PER_TILE = TILE_N / R;
     constexpr bool WHOLE = (R == TILE_N);                  // whole blobs: weights, scales and zero points in one bulk copy
     constexpr int ZB = R / 2 < 16 ? 16 : R / 2;            // bytes of zero points fetched per group (16-byte granules)
     constexpr uint32_t STAGE_BYTES = st_stage_bytes(MB, RBLK);
     constexpr uint32_t ACT_BYTES = GS * MP * GROUP;
-    constexpr uint32_t NARROW_W_BYTES = 16384 + GS * 2 * R + GS * ZB;
+    constexpr uint32_t NARROW_W_BYTES = ST_NIB_BYTES + GS * 2 * R + GS * ZB;
     // byte offsets inside a stage
     constexpr int NIB_G = WHOLE ? BLOB_BYTES : R * 64;               // from one group's rows to the next group's
-    constexpr int SC_BASE = WHOLE ? BLOB_SCALE_OFF : 16384, SC_G = WHOLE ? BLOB_BYTES : 2 * R;
-    constexpr int Z_BASE = WHOLE ? BLOB_ZERO_OFF : 16384 + GS * 2 * R, Z_G = WHOLE ? BLOB_BYTES : ZB;
-    static_assert(NARROW_W_BYTES <= ST_W_BYTES && 2 * BLOB_BYTES <= ST_W_BYTES, "weight part of a stage");
+    constexpr int SC_BASE = WHOLE ? BLOB_SCALE_OFF : ST_NIB_BYTES, SC_G = WHOLE ? BLOB_BYTES : 2 * R;
+    constexpr int Z_BASE = WHOLE ? BLOB_ZERO_OFF : ST_NIB_BYTES + GS * 2 * R, Z_G = WHOLE ? BLOB_BYTES : ZB;
+    static_assert(NARROW_W_BYTES <= ST_W_BYTES && (ST_UNITS / 8) * BLOB_BYTES <= ST_W_BYTES, "weight part of a stage");
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -567,7 +573,7 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
 template <int MB, int RBLK, bool DEBUG>
 cudaError_t launch_strip(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed, void* y,
                          int M, int N, int K, int ctas, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
-    constexpr int R = 16 * RBLK, GS = 16 / RBLK, MP = 8 * MB;
+    constexpr int R = 16 * RBLK, GS = ST_UNITS / RBLK, MP = 8 * MB;
     const int G = K / GROUP;
     const int fixed = st_layout(MB, RBLK, 0, G).total + 1024;
     int stages = (ST_SMEM_BUDGET - fixed) / st_stage_bytes(MB, RBLK);
