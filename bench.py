@@ -353,26 +353,34 @@ def run_large_m_roofline(torch, B, peaks, l2_bytes, timer):
 
 
 def run_quantize_roofline(torch, B, peaks, l2_bytes, timer):
-    """quantize_act alone at 1024 x 4096 on inputs visited in turn (more than two L2 capacities in all)."""
-    M, K = 1024, 4096
-    nbytes = wl.algorithmic_bytes_quantize(M, K)
-    ncopies = copies_for(2 * M * K, l2_bytes)
-    xs = [torch.randn((M, K), device="cuda").to(torch.bfloat16) for _ in range(ncopies)]
-    qa = torch.empty((M, K), dtype=torch.int8, device="cuda")
-    sa = torch.empty((M,), dtype=torch.float16, device="cuda")
-    asum = torch.empty((M, K // 128), dtype=torch.int32, device="cuda")
+    """quantize_act alone at 1024 x 4096 (one wave of CTAs: latency shows) and 4096 x 4096 (several waves), on inputs
+    visited in turn (more than two L2 capacities in all)."""
+    def one(M, K):
+        nbytes = wl.algorithmic_bytes_quantize(M, K)
+        ncopies = copies_for(2 * M * K, l2_bytes)
+        xs = [torch.randn((M, K), device="cuda").to(torch.bfloat16) for _ in range(ncopies)]
+        qa = torch.empty((M, K), dtype=torch.int8, device="cuda")
+        sa = torch.empty((M,), dtype=torch.float16, device="cuda")
+        asum = torch.empty((M, K // 128), dtype=torch.int32, device="cuda")
 
-    def body():
-        for x in xs:
-            B.w4a8_quantize_act(x, 128, out=(qa, sa, asum))
-    _, times = timer.graph_ms(body, replays=5, warm=2)
-    us = float(np.median(times)) * 1e3 / ncopies
+        def body():
+            for x in xs:
+                B.w4a8_quantize_act(x, 128, out=(qa, sa, asum))
+        _, times = timer.graph_ms(body, replays=5, warm=2)
+        us = float(np.median(times)) * 1e3 / ncopies
+        del xs
+        torch.cuda.empty_cache()
+        return nbytes, us
+    nbytes, us = one(1024, 4096)
     gbs = nbytes / us / 1e3
-    del xs
-    torch.cuda.empty_cache()
-    return {"bound": "hbm", "kernel": "quantize_act_kernel<256>", "workload": f"M={M} K={K}", "achieved": round(gbs, 1),
+    nbytes4, us4 = one(4096, 4096)
+    gbs4 = nbytes4 / us4 / 1e3
+    return {"bound": "hbm", "kernel": "quantize_act_kernel<256 threads, 2 chunks, reciprocal + tie fallback>",
+            "workload": "M=1024 K=4096", "achieved": round(gbs, 1),
             "unit": "GB/s", "peak": peaks["hbm_gbs"], "frac": round(gbs / peaks["hbm_gbs"], 4), "us_per_launch": round(us, 2),
-            "algorithmic_bytes_per_launch": nbytes, "traffic": 8427520,
+            "algorithmic_bytes_per_launch": nbytes, "traffic": QUANTIZE_TRAFFIC_BYTES_PER_LAUNCH,
+            "m4096": {"workload": "M=4096 K=4096", "achieved": round(gbs4, 1), "frac": round(gbs4 / peaks["hbm_gbs"], 4),
+                      "us_per_launch": round(us4, 2), "algorithmic_bytes_per_launch": nbytes4},
             "timing": "median of 5 replays of back-to-back launches in one graph"}
 
 
@@ -665,6 +673,7 @@ def run_shape(args):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one GEMM launch at the headline shape, by kernel, from the ncu
 # captures summarised under profiles/ (gemm_strip_qkv_M8.md, gemm_cluster_qkv_M8.md)
+QUANTIZE_TRAFFIC_BYTES_PER_LAUNCH = 8427520      # ncu, quantize_act at 1024 x 4096 (profiles/quantize_act_M1024_K4096.md)
 TRAFFIC_BYTES_PER_LAUNCH = {"gemm_strip_kernel": 13148416, "gemm_cluster_kernel": 13144832}
 E2E_DEPTH = int(os.environ.get("W4A8_E2E_DEPTH", "4"))          # host requests in flight in the end-to-end measurement
 
