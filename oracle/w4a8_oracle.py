@@ -114,6 +114,30 @@ def w4a8_linear(x_bits, qw, sw_bits, z, group):
     return dict(qa=qa, sa=sa_bits, asum=asum, D=D, ref=ref)
 
 
+# ---- the step after the fused gate+up projection (Sec. 3.5, "Kernel Fusion") -----------------
+def silu_mul(y_gate_bits, y_up_bits):
+    """h[m,c] = bf16_rne( SiLU(gate[m,c]) * up[m,c] ),  SiLU(v) = v / (1 + exp(-v)),  in fp64.
+
+    gate and up are the two halves of the fused gate+up projection's bf16 output (Sec. 3.5 fuses
+    the two projections into one GEMM and merges the element-wise operations that follow), given
+    here as two separate [M,I] arrays of bf16 bit patterns: how a kernel lays the two halves out
+    in one buffer is not this function's business.  Returns (h fp64 before the rounding, h bf16 bits).
+    """
+    g = bf16_bits_to_f64(y_gate_bits)
+    u = bf16_bits_to_f64(y_up_bits)
+    with np.errstate(over="ignore"):
+        h = g / (1.0 + np.exp(-g)) * u
+    return h, f64_to_bf16_bits(h)
+
+
+def silu_mul_quantize(y_gate_bits, y_up_bits, group):
+    """The down projection's quantised input from the gate+up projection's output:
+    quantize_act(silu_mul(gate, up)).  Returns dict(h, h_bits, qa, sa, asum)."""
+    h, h_bits = silu_mul(y_gate_bits, y_up_bits)
+    qa, sa_bits, asum = quantize_act(h_bits, group)
+    return dict(h=h, h_bits=h_bits, qa=qa, sa=sa_bits, asum=asum)
+
+
 # ---- acceptance band for a bf16 result ------------------------------------------------
 def tolerance(ref):
     """Per-element bound 2^-7 |ref| + 1e-3 rms(ref), rms over the whole [M,N] result."""

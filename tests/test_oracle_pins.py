@@ -372,3 +372,86 @@ def test_tolerance_band():
     bad = onp.f64_to_bf16_bits(ref * 1.05)
     ok, ratio = onp.within_tolerance(bad, ref)
     assert not ok and ratio > 1
+
+
+# ---- SiLU(gate) * up and the requantisation that follows (Sec. 3.5, "Kernel Fusion") ----------------
+def read_silu_golden():
+    rows = []
+    import os
+    with open(os.path.join(os.path.dirname(__file__), "golden", "silu_mul_examples.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            g, u, prod, h = line.split()
+            rows.append((int(g, 16), int(u, 16), float(prod), int(h, 16)))
+    return rows
+
+
+def test_silu_mul_matches_hand_worked_examples():
+    rows = read_silu_golden()
+    g = np.array([[r[0] for r in rows]], dtype=np.uint16)
+    u = np.array([[r[1] for r in rows]], dtype=np.uint16)
+    h, h_bits = onp.silu_mul(g, u)
+    assert np.allclose(h[0], [r[2] for r in rows], rtol=0, atol=6e-11)
+    assert h_bits[0].tolist() == [r[3] for r in rows]
+
+
+def test_silu_mul_against_library_routines_and_identities():
+    import torch
+    from scipy.special import expit
+    rng = np.random.default_rng(5)
+    gb = wl.f32_to_bf16_bits((rng.standard_normal((7, 64)) * 6).astype(np.float32))
+    ub = wl.f32_to_bf16_bits((rng.standard_normal((7, 64)) * 3).astype(np.float32))
+    g, u = onp.bf16_bits_to_f64(gb), onp.bf16_bits_to_f64(ub)
+    h, h_bits = onp.silu_mul(gb, ub)
+    # SiLU(v) = v * logistic(v): scipy's logistic function and torch's silu, both in fp64
+    assert np.allclose(h, g * expit(g) * u, rtol=1e-14, atol=0)
+    assert np.allclose(h, (torch.nn.functional.silu(torch.from_numpy(g)) * torch.from_numpy(u)).numpy(), rtol=1e-14, atol=0)
+    # SiLU(v) - SiLU(-v) = v, with up = 1 (bit pattern 0x3F80) and the sign bit of gate flipped
+    one = np.full_like(gb, 0x3F80)
+    hp, _ = onp.silu_mul(gb, one)
+    hm, _ = onp.silu_mul(gb ^ np.uint16(0x8000), one)
+    assert np.allclose(hp - hm, g, rtol=1e-14, atol=1e-300)
+    # exact linearity in up for powers of two, oddness in up, zero gate -> zero
+    h2, _ = onp.silu_mul(gb, wl.f32_to_bf16_bits((onp.bf16_bits_to_f64(ub) * 4.0).astype(np.float32)))
+    assert np.array_equal(h2, 4.0 * h)
+    hn, hn_bits = onp.silu_mul(gb, ub ^ np.uint16(0x8000))
+    assert np.array_equal(hn, -h) and np.array_equal(hn_bits, h_bits ^ np.uint16(0x8000))
+    hz, hz_bits = onp.silu_mul(np.zeros_like(gb), ub)
+    assert not hz.any() and not (hz_bits & 0x7FFF).any()
+    # far out the function is the identity on one side and zero on the other; no overflow to NaN at -90 (exp(90) is finite
+    # in fp64) nor at the largest bf16 magnitudes
+    big = wl.f32_to_bf16_bits(np.array([[40.0, -40.0, 90.0, -90.0, 3.0e38, -3.0e38]], dtype=np.float32))
+    hb, hb_bits = onp.silu_mul(big, np.full_like(big, 0x3F80))
+    assert hb[0, 0] == 40.0 and abs(hb[0, 1]) < 1e-15 and hb[0, 2] == 90.0 and abs(hb[0, 3]) < 1e-37
+    assert hb[0, 4] == onp.bf16_bits_to_f64(big)[0, 4] and hb[0, 5] == 0.0 and np.all(np.isfinite(hb))
+    # the rounding is the pinned bf16 rounding of the fp64 value
+    assert np.array_equal(h_bits, onp.f64_to_bf16_bits(h))
+
+
+def test_silu_mul_quantize_is_the_quantiser_on_h():
+    rng = np.random.default_rng(6)
+    gb = wl.f32_to_bf16_bits((rng.standard_normal((3, 256)) * 4).astype(np.float32))
+    ub = wl.f32_to_bf16_bits((rng.standard_normal((3, 256)) * 2).astype(np.float32))
+    gb[1] = 0                                                   # a token whose h is all zero: scale 0, codes 0
+    r = onp.silu_mul_quantize(gb, ub, 128)
+    h = onp.bf16_bits_to_f64(r["h_bits"])
+    sa = onp.fp16_bits_to_f64(r["sa"])
+    assert sa[1] == 0.0 and not r["qa"][1].any()
+    for m in (0, 2):
+        # the a-priori statement of the quantiser: |h - sa q| <= sa / 2 wherever nothing was clamped, and the largest
+        # magnitude maps to +-127
+        assert np.all(np.abs(h[m] - sa[m] * r["qa"][m]) <= sa[m] / 2 + 1e-12)
+        assert np.abs(r["qa"][m]).max() == 127
+    assert np.array_equal(r["asum"], r["qa"].astype(np.int64).reshape(3, 2, 128).sum(axis=2))
+    # worked example through the golden fixture: the six h values as one token (padded to a group of 8)
+    rows = read_silu_golden()
+    g8 = np.array([[r_[0] for r_ in rows] + [0, 0]], dtype=np.uint16)
+    u8 = np.array([[r_[1] for r_ in rows] + [0, 0]], dtype=np.uint16)
+    q = onp.silu_mul_quantize(g8, u8, 8)
+    # amax = 2.1875 -> sa = fp16(2.1875 / 127 = 0.017224409...) ; fp16 step in [2^-6, 2^-5) is 2^-16: 1128.82 -> 1129 * 2^-16
+    assert onp.fp16_bits_to_f64(q["sa"])[0] == 1129 * 2.0 ** -16
+    # codes: h / sa = 126.98, -51.02, -125.16, 0, 18.03, -0.156 -> 127, -51, -125, 0, 18, 0
+    assert q["qa"][0].tolist() == [127, -51, -125, 0, 18, 0, 0, 0]
+    assert q["asum"][0].tolist() == [127 - 51 - 125 + 18]
