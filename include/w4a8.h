@@ -155,6 +155,52 @@ typedef struct {
 w4a8_status w4a8_plan(int M, int N, int K, int group, w4a8_plan_info* out);
 
 /*
+ * The step after the fused gate+up projection (Sec. 3.5, "Kernel Fusion": gate and up are one GEMM, and
+ * the element-wise operations that follow are merged into their neighbours): from the projection's
+ * output to the quantised input of the down projection, h never making a round trip as a separate pass.
+ *
+ *   h[m,c]  = bf16_rne( SiLU(gate[m,c]) * up[m,c] ),  SiLU(v) = v / (1 + exp(-v)),  gate and up the bf16
+ *             outputs of the projection; evaluated in fp32 with the fast exponential (h equals the exactly
+ *             computed value or its bf16 neighbour)
+ *   (qa_h, sa_h, asum_h) = the activation quantisation of w4a8_quantize_act applied to h (bit-exact
+ *             given h): the operands w4a8_gemm takes for the down projection.
+ *
+ * Channel layout of the fused layer (this library's reading; the paper gives none): its N = 2 I output
+ * channels alternate in runs of eight - channel n = 16 b + i is gate channel 8 b + i for i < 8 and up
+ * channel 8 b + i - 8 for i >= 8.  A 16-byte piece of an output row is thus eight gate values or the eight
+ * up values of the same indices, and the gate and up of one channel meet in one thread of the GEMM's
+ * epilogue.  The caller orders the rows of the two weight matrices so before w4a8_pack_weights; the
+ * packed format itself is unchanged.
+ *
+ * w4a8_silu_mul_quantize: the step alone, for a projection output that is already in memory.
+ *   y_gate_up  device, bf16 [M, 2 I] in the layout above (16-byte aligned)
+ *   h          device, bf16 [M, I], receives h; may be NULL
+ *   qa_h       device, int8 [M, I]; sa_h fp16 [M]; asum_h int32 [M, I / 128]
+ *   I % 128 == 0, group == 128.  One kernel, one CTA per token.
+ *
+ * w4a8_gate_up_silu_quantize: projection and step together.  Where w4a8_gemm would take the strip kernel
+ * (w4a8_gate_up_is_one_kernel returns 1: up to 8 tokens, and 9..16 on wide layers) this is ONE kernel: the
+ * strip kernel's epilogue forms h from its own sums, the CTAs meet at a grid-wide barrier (bounded wait; the
+ * grid is sized so that every CTA is resident), and all warps then quantise h; y is never stored.  Otherwise
+ * it is w4a8_gemm into y_scratch followed by w4a8_silu_mul_quantize, with identical results.
+ *   qa, sa, asum, packed_gate_up, M, N (= 2 I), K, group, workspace: as for w4a8_gemm
+ *   h          device, bf16 [M, I]: output, and in the one-kernel form also the buffer through which the
+ *              CTAs exchange h (required)
+ *   y_scratch  device, bf16 [M, N]; needed only when w4a8_gate_up_is_one_kernel returns 0, else may be NULL
+ * Errors as for w4a8_gemm, W4A8_ERR_SHAPE also for I % 128 != 0.  The one-kernel form keeps 18 words of the
+ * workspace header (per-token maxima and two counters) that it leaves zero; after W4A8_ERR_TIMEOUT the
+ * workspace must be initialised again before its next use.
+ */
+w4a8_status w4a8_silu_mul_quantize(const void* y_gate_up_bf16, int M, int I, int group, void* h_bf16,
+                                   int8_t* qa_h, uint16_t* sa_h, int32_t* asum_h, void* stream);
+int w4a8_gate_up_is_one_kernel(int M, int N, int K, int group);
+w4a8_status w4a8_gate_up_silu_quantize(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
+                                       const void* packed_gate_up, int M, int N, int K, int group,
+                                       void* h_bf16, int8_t* qa_h, uint16_t* sa_h, int32_t* asum_h,
+                                       void* y_scratch_bf16, void* workspace, size_t workspace_bytes,
+                                       void* stream);
+
+/*
  * Variant for weights whose scale does not change along K (per-channel scales: the paper does not
  * give its group size, Sec. 3.4; this is the coarsest choice, group 128 the library's default).
  * Same packed format and the same per-group zero points; the caller guarantees that the scales of

@@ -21,7 +21,8 @@ WORKSPACE_ZEROED_BYTES = 4096 + 192 * 16384
 EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w4a8_workspace_init",
            "w4a8_pack_weights", "w4a8_unpack_weights", "w4a8_quantize_act", "w4a8_gemm", "w4a8_gemm_path",
            "w4a8_linear", "w4a8_linear_host", "w4a8_gemm_static_scratch", "w4a8_check_status", "w4a8_plan",
-           "w4a8_gemm_per_channel", "w4a8_static_scratch_status", "w4a8_selftest_wait_timeout")
+           "w4a8_gemm_per_channel", "w4a8_static_scratch_status", "w4a8_selftest_wait_timeout",
+           "w4a8_silu_mul_quantize", "w4a8_gate_up_is_one_kernel", "w4a8_gate_up_silu_quantize")
 
 _lib = None
 
@@ -63,6 +64,12 @@ def lib():
         L.w4a8_gemm_per_channel.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp, vp]
         L.w4a8_plan.restype = ci
         L.w4a8_plan.argtypes = [ci, ci, ci, ci, vp]
+        L.w4a8_silu_mul_quantize.restype = ci
+        L.w4a8_silu_mul_quantize.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp]
+        L.w4a8_gate_up_is_one_kernel.restype = ci
+        L.w4a8_gate_up_is_one_kernel.argtypes = [ci, ci, ci, ci]
+        L.w4a8_gate_up_silu_quantize.restype = ci
+        L.w4a8_gate_up_silu_quantize.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, sz, vp]
         L.w4a8_linear.restype = ci
         L.w4a8_linear.argtypes = [vp, vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, sz, vp]
         L.w4a8_linear_host.restype = ci
@@ -199,6 +206,55 @@ def w4a8_gemm_per_channel(qa, sa, packed_w, N, workspace, group=GROUP, out=None,
                                        _ptr(workspace), workspace.numel(), _ptr(debug_sums), _stream(stream)),
            "w4a8_gemm_per_channel")
     return out
+
+
+def gate_up_row_order(I):
+    """Row order of the fused gate+up layer: entry n is the row of the concatenation [gate rows; up rows] (2 I rows)
+    that becomes output channel n - runs of eight gate channels alternating with the eight up channels of the same
+    indices (see w4a8_gate_up_silu_quantize in the header).  Index arithmetic only."""
+    import numpy as np
+    n = np.arange(2 * I)
+    b, i = n // 16, n % 16
+    return np.where(i < 8, 8 * b + i, I + 8 * b + i - 8)
+
+
+def _h_outputs(M, I, group, device, out):
+    if out is not None:
+        return out
+    return (torch.empty((M, I), dtype=torch.bfloat16, device=device), torch.empty((M, I), dtype=torch.int8, device=device),
+            torch.empty((M,), dtype=torch.float16, device=device), torch.empty((M, I // group), dtype=torch.int32, device=device))
+
+
+def w4a8_silu_mul_quantize(y_gate_up, group=GROUP, out=None, stream=None):
+    """y bf16 [M, 2 I] of a fused gate+up layer -> (h bf16 [M,I], qa_h int8 [M,I], sa_h fp16 [M], asum_h int32 [M,I/group])."""
+    _dev(y_gate_up, torch.bfloat16, "y_gate_up")
+    M, N = y_gate_up.shape
+    I = N // 2
+    h, qa_h, sa_h, asum_h = _h_outputs(M, I, group, y_gate_up.device, out)
+    _check(lib().w4a8_silu_mul_quantize(_ptr(y_gate_up), M, I, group, _ptr(h), _ptr(qa_h), _ptr(sa_h), _ptr(asum_h),
+                                        _stream(stream)), "w4a8_silu_mul_quantize")
+    return h, qa_h, sa_h, asum_h
+
+
+def w4a8_gate_up_is_one_kernel(M, N, K, group=GROUP):
+    return bool(lib().w4a8_gate_up_is_one_kernel(M, N, K, group))
+
+
+def w4a8_gate_up_silu_quantize(qa, sa, asum, packed_gate_up, N, workspace, group=GROUP, y_scratch=None, out=None, stream=None):
+    """Fused gate+up projection, SiLU(gate) * up and the down projection's activation quantisation: one kernel where
+    w4a8_gemm would take the strip kernel, else the GEMM into y_scratch followed by w4a8_silu_mul_quantize."""
+    _dev(qa, torch.int8, "qa"), _dev(sa, torch.float16, "sa"), _dev(asum, torch.int32, "asum")
+    _dev(packed_gate_up, torch.uint8, "packed_gate_up"), _dev(workspace, torch.uint8, "workspace")
+    M, K = qa.shape
+    I = N // 2
+    h, qa_h, sa_h, asum_h = _h_outputs(M, I, group, qa.device, out)
+    if y_scratch is None and M > 0 and not w4a8_gate_up_is_one_kernel(M, N, K, group):
+        y_scratch = torch.empty((M, N), dtype=torch.bfloat16, device=qa.device)
+    _check(lib().w4a8_gate_up_silu_quantize(_ptr(qa), _ptr(sa), _ptr(asum), _ptr(packed_gate_up), M, N, K, group,
+                                            _ptr(h), _ptr(qa_h), _ptr(sa_h), _ptr(asum_h), _ptr(y_scratch),
+                                            _ptr(workspace), workspace.numel(), _stream(stream)),
+           "w4a8_gate_up_silu_quantize")
+    return h, qa_h, sa_h, asum_h
 
 
 class PlanInfo(ctypes.Structure):

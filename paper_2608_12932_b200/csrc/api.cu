@@ -186,6 +186,51 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
     return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
 
+w4a8_status w4a8_silu_mul_quantize(const void* y_gate_up_bf16, int M, int I, int group, void* h_bf16,
+                                   int8_t* qa_h, uint16_t* sa_h, int32_t* asum_h, void* stream) {
+    if (group != GROUP || I <= 0 || I % GROUP != 0 || M < 0) return W4A8_ERR_SHAPE;
+    if (M == 0) return W4A8_OK;
+    if (!y_gate_up_bf16 || !qa_h || !sa_h || !asum_h) return W4A8_ERR_NULL;
+    if (!aligned(y_gate_up_bf16, 16) || !aligned(qa_h, 16) || !aligned(sa_h, 2) || !aligned(asum_h, 4) ||
+        (h_bf16 && !aligned(h_bf16, 16)))
+        return W4A8_ERR_ALIGN;
+    w4a8_status a = arch_check();
+    if (a != W4A8_OK) return a;
+    return launch_silu_mul_quantize(y_gate_up_bf16, M, I, h_bf16, qa_h, sa_h, asum_h, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+int w4a8_gate_up_is_one_kernel(int M, int N, int K, int group) {
+    if (!shape_ok(N, K, group) || M < 1 || (N / 2) % GROUP != 0) return 0;
+    return auto_takes_strip(M, N, K) ? 1 : 0;
+}
+
+w4a8_status w4a8_gate_up_silu_quantize(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed_gate_up,
+                                       int M, int N, int K, int group, void* h_bf16, int8_t* qa_h, uint16_t* sa_h,
+                                       int32_t* asum_h, void* y_scratch_bf16, void* workspace, size_t workspace_bytes,
+                                       void* stream) {
+    if (!shape_ok(N, K, group) || M < 0 || (N / 2) % GROUP != 0) return W4A8_ERR_SHAPE;
+    if (M == 0) return W4A8_OK;
+    if (!qa || !sa || !asum || !packed_gate_up || !h_bf16 || !qa_h || !sa_h || !asum_h || !workspace) return W4A8_ERR_NULL;
+    const bool one = w4a8_gate_up_is_one_kernel(M, N, K, group) != 0;
+    if (!one && !y_scratch_bf16) return W4A8_ERR_NULL;
+    if (!aligned(qa, 16) || !aligned(sa, 2) || !aligned(asum, 4) || !aligned(packed_gate_up, 128) || !aligned(h_bf16, 16) ||
+        !aligned(qa_h, 16) || !aligned(sa_h, 2) || !aligned(asum_h, 4) || !aligned(workspace, 256) ||
+        (y_scratch_bf16 && !aligned(y_scratch_bf16, 16)))
+        return W4A8_ERR_ALIGN;
+    if (workspace_bytes < w4a8_workspace_bytes(M, N, K, group)) return W4A8_ERR_WORKSPACE;
+    w4a8_status a = arch_check();
+    if (a != W4A8_OK) return a;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (one)
+        return launch_gemm_strip_gate_up(qa, sa, asum, packed_gate_up, M, N, K, h_bf16, qa_h, sa_h, asum_h, workspace, st) == cudaSuccess
+                   ? W4A8_OK : W4A8_ERR_CUDA;
+    w4a8_status g = w4a8_gemm_path(W4A8_PATH_AUTO, qa, sa, asum, packed_gate_up, y_scratch_bf16, M, N, K, group, workspace,
+                                   workspace_bytes, nullptr, stream);
+    if (g != W4A8_OK) return g;
+    return launch_silu_mul_quantize(y_scratch_bf16, M, N / 2, h_bf16, qa_h, sa_h, asum_h, st) == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
 w4a8_status w4a8_gemm_per_channel(const int8_t* qa, const uint16_t* sa, const void* packed_w, void* y_bf16,
                                   int M, int N, int K, int group, void* workspace, size_t workspace_bytes,
                                   int32_t* debug_sums, void* stream) {

@@ -47,6 +47,7 @@
 #include <cstdlib>
 #endif
 #include "ptx_sm100.cuh"
+#include "quant_common.cuh"
 #include "w4a8_internal.cuh"
 
 namespace w4a8 {
@@ -149,9 +150,23 @@ struct StripArgs {
     uint32_t* status;
     unsigned long long* slots;   // one strip of tagged fp32 sums per CTA (STRIP_SLOT_BYTES each), zero between calls
     int32_t* debug_partials;
+    // fused form only (gate+up projection -> SiLU * up -> requantise): N = 2 I
+    __nv_bfloat16* h;        // [M, I] bf16, written before and read after the grid-wide barrier
+    int8_t* qa_h;            // [M, I]
+    uint16_t* sa_h;          // [M]
+    int32_t* asum_h;         // [M, I / 128]
+    uint32_t* sync;          // workspace words: amax[16] (bf16 magnitudes), arrivals, departures; zero between calls
 };
 
-template <int MB, int RBLK, bool DEBUG>
+// FUSE (Sec. 3.5, "Kernel Fusion"): the layer is a fused gate+up projection whose output channels alternate in
+// runs of eight (rows 16 b .. 16 b + 7 of the packed layer are gate channels 8 b .. 8 b + 7, rows 16 b + 8 .. 16 b + 15
+// the up channels of the same indices), so that a lane of the epilogue warp holds gate and up of one channel.  The
+// epilogue rounds both to bf16 as the plain kernel would, computes h = bf16(SiLU(gate) * up), stores h and keeps
+// the largest |h| per token; all CTAs then meet at a grid-wide barrier (every CTA of the grid is resident: the
+// launcher bounds the grid by the occupancy), after which the warps of all CTAs quantise h, one (token, group of
+// 128) per warp: codes, token scales and group sums of the down projection's input leave this kernel; y is never
+// stored.
+template <int MB, int RBLK, bool DEBUG, bool FUSE>
 __global__ void __launch_bounds__(ST_THREADS, 2)
 gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_nib,
                   const __grid_constant__ CUtensorMap tm_scale, const __grid_constant__ CUtensorMap tm_zero,
@@ -472,6 +487,10 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
         ulonglong2* mine = reinterpret_cast<ulonglong2*>(reinterpret_cast<uint8_t*>(a.slots) + (size_t)blockIdx.x * SLOT);
         ulonglong2* theirs = reinterpret_cast<ulonglong2*>(reinterpret_cast<uint8_t*>(a.slots) + (size_t)(blockIdx.x + 1) * SLOT);
         constexpr unsigned long long TAG = 1ull << 32;
+        constexpr int HPITCH = R + 16;                            // fused form: bytes per token row of the staged h (R / 2 channels)
+        uint32_t hmax[MB][2];                                     // fused form: largest |h| (bf16 bits) of this lane's tokens
+#pragma unroll
+        for (int mb = 0; mb < MB; ++mb) hmax[mb][0] = hmax[mb][1] = 0u;
         for (int q = 0; q < nseg && ok; ++q) {
             const int strip = first_strip + q;
             const bool has_start = lo <= strip * sps, has_end = hi >= (strip + 1) * sps;
@@ -540,6 +559,17 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
                 const uint32_t yo = ystage + m0 * YPITCH + (rb * 16 + r) * 2;
                 const __nv_bfloat16 o0 = __float2bfloat16_rn(acc.x * t0), o1 = __float2bfloat16_rn(acc.y * t1);
                 const __nv_bfloat16 o2 = __float2bfloat16_rn(acc.z * t0), o3 = __float2bfloat16_rn(acc.w * t1);
+                if (FUSE) {
+                    // (o0, o2) = (gate, up) of channel 8 rb + r for token m0, (o1, o3) for token m0 + 1
+                    const uint32_t h0 = silu_mul_bf16_bits(__bfloat162float(o0), __bfloat162float(o2));
+                    const uint32_t h1 = silu_mul_bf16_bits(__bfloat162float(o1), __bfloat162float(o3));
+                    hmax[mb][0] = max(hmax[mb][0], h0 & 0x7FFFu);
+                    hmax[mb][1] = max(hmax[mb][1], h1 & 0x7FFFu);
+                    const uint32_t ho = ystage + m0 * HPITCH + (rb * 8 + r) * 2;
+                    asm volatile("st.shared.u16 [%0], %1;" ::"r"(ho), "h"((unsigned short)h0) : "memory");
+                    asm volatile("st.shared.u16 [%0], %1;" ::"r"(ho + HPITCH), "h"((unsigned short)h1) : "memory");
+                    continue;
+                }
                 asm volatile("st.shared.u16 [%0], %1;" ::"r"(yo), "h"(__bfloat16_as_ushort(o0)) : "memory");
                 asm volatile("st.shared.u16 [%0], %1;" ::"r"(yo + YPITCH), "h"(__bfloat16_as_ushort(o1)) : "memory");
                 asm volatile("st.shared.u16 [%0], %1;" ::"r"(yo + 16), "h"(__bfloat16_as_ushort(o2)) : "memory");
@@ -547,7 +577,7 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
             }
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(part_empty);
-            if (has_start) {
+            if (has_start && !FUSE) {
                 // the strip leaves in 16-byte pieces: R / 8 per token row
                 constexpr int CPR = R / 8;
                 for (int c = lane; c < a.M * CPR; c += 32) {
@@ -557,10 +587,90 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
                 }
                 __syncwarp();
             }
+            if (has_start && FUSE) {
+                // the strip's R / 2 channels of h, 16-byte pieces
+                constexpr int CPR = R / 16;
+                const int I = a.N / 2;
+                for (int c = lane; c < a.M * CPR; c += 32) {
+                    const int m = c / CPR, col = c - m * CPR;
+                    const uint4 v = ptx::lds128(ystage + m * HPITCH + col * 16);
+                    *reinterpret_cast<uint4*>(a.h + (size_t)m * I + (size_t)strip * (R / 2) + col * 8) = v;
+                }
+                __syncwarp();
+            }
+        }
+        if (FUSE) {
+            // largest |h| per token over this CTA's strips: lanes of equal j hold the same two tokens
+#pragma unroll
+            for (int mb = 0; mb < MB; ++mb)
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    uint32_t v = hmax[mb][t];
+                    v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, 4));
+                    v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, 8));
+                    v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, 16));
+                    const int m = 8 * mb + 2 * j + t;
+                    if (r == 0 && m < a.M && v != 0u) atomicMax(a.sync + m, v);
+                }
+            __threadfence();                                   // h and the maxima before the arrival
+            __syncwarp();
+            if (lane == 0) atomicAdd(a.sync + 16, 1u);
         }
         if (lane == 0) ST_STAMP(6);
     }
     __syncwarp();
+    if (FUSE) {
+        // ---- grid-wide barrier, then the requantisation of h by all warps of all CTAs ----
+        __syncthreads();
+        if (tid == 0) {
+            uint64_t t0 = 0;
+            for (uint32_t spin = 0; !*abort_flag; ++spin) {
+                uint32_t v;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a.sync + 16) : "memory");
+                if (v >= gridDim.x) break;
+                if ((spin & 15) == 15) {
+                    const uint64_t now = ptx::globaltimer_ns();
+                    if (t0 == 0) t0 = now;
+                    else if (now - t0 > ptx::WAIT_LIMIT_NS) { *abort_flag = 1; break; }
+                }
+                __nanosleep(100);
+            }
+            __threadfence();
+        }
+        __syncthreads();
+        if (!*abort_flag) {
+            const int I = a.N / 2, Gh = I / GROUP;
+            constexpr int WARPS = ST_THREADS / 32;
+            for (int u = blockIdx.x * WARPS + warp; u < a.M * Gh; u += gridDim.x * WARPS) {
+                const int m = u / Gh, g = u - m * Gh;
+                const __half sh = row_scale_from_amax_bits(__ldcg(a.sync + m));
+                const float s = __half2float(sh);
+                const size_t at = (size_t)m * I + (size_t)g * GROUP + 4 * lane;
+                const uint2 hv = __ldcg(reinterpret_cast<const uint2*>(a.h + at));
+                int q0 = 0, q1 = 0, q2 = 0, q3 = 0;
+                if (s != 0.0f) {
+                    q0 = quant1(hv.x << 16, s); q1 = quant1(hv.x & 0xFFFF0000u, s);
+                    q2 = quant1(hv.y << 16, s); q3 = quant1(hv.y & 0xFFFF0000u, s);
+                }
+                *reinterpret_cast<uint32_t*>(a.qa_h + at) =
+                    (uint32_t)(q0 & 0xFF) | ((uint32_t)(q1 & 0xFF) << 8) | ((uint32_t)(q2 & 0xFF) << 16) | ((uint32_t)q3 << 24);
+                const int sum = __reduce_add_sync(0xFFFFFFFFu, q0 + q1 + q2 + q3);
+                if (lane == 0) {
+                    a.asum_h[(size_t)m * Gh + g] = sum;
+                    if (g == 0) a.sa_h[m] = __half_as_ushort(sh);
+                }
+            }
+        }
+        __syncthreads();
+        // the last CTA to leave puts the words back to zero for the next call
+        if (tid == 0) {
+            const uint32_t old = atomicAdd(a.sync + 17, 1u);
+            if (old == gridDim.x - 1) {
+                for (int i = 0; i < 18; ++i) a.sync[i] = 0u;
+                __threadfence();
+            }
+        }
+    }
     if (*abort_flag) {
         if (lane == 0) atomicExch(a.status, (uint32_t)W4A8_ERR_TIMEOUT);
         // copies that were requested may still be in flight: give them a bounded time to land before the
@@ -570,9 +680,17 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
     }
 }
 
-template <int MB, int RBLK, bool DEBUG>
+struct FuseOut {
+    void* h;
+    int8_t* qa_h;
+    uint16_t* sa_h;
+    int32_t* asum_h;
+};
+
+template <int MB, int RBLK, bool DEBUG, bool FUSE>
 cudaError_t launch_strip(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed, void* y,
-                         int M, int N, int K, int ctas, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
+                         int M, int N, int K, int ctas, void* workspace, int32_t* debug_partials, const FuseOut* fuse,
+                         cudaStream_t stream) {
     constexpr int R = 16 * RBLK, GS = ST_UNITS / RBLK, MP = 8 * MB;
     const int G = K / GROUP;
     const int fixed = st_layout(MB, RBLK, 0, G).total + 1024;
@@ -585,10 +703,20 @@ cudaError_t launch_strip(const int8_t* qa, const uint16_t* sa, const int32_t* as
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     static bool attr_done[64] = {false};
+    static int resident[64] = {0};                          // CTAs of this instance that fit on the device at once
     if (!attr_done[dev]) {
-        e = cudaFuncSetAttribute(gemm_strip_kernel<MB, RBLK, DEBUG>, cudaFuncAttributeMaxDynamicSharedMemorySize, ST_SMEM_BUDGET);
+        e = cudaFuncSetAttribute(gemm_strip_kernel<MB, RBLK, DEBUG, FUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, ST_SMEM_BUDGET);
         if (e != cudaSuccess) return e;
+        int per_sm = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, gemm_strip_kernel<MB, RBLK, DEBUG, FUSE>, ST_THREADS, ST_SMEM_BUDGET);
+        if (e != cudaSuccess) return e;
+        resident[dev] = per_sm * device_sm_count();
         attr_done[dev] = true;
+    }
+    if (FUSE) {
+        // the grid-wide barrier needs every CTA resident at the same time
+        if (resident[dev] < 1) return cudaErrorInvalidConfiguration;
+        if (ctas > resident[dev]) ctas = resident[dev];
     }
     CUtensorMap tm_act, tm_nib, tm_scale, tm_zero;
     e = make_qa_group_map(&tm_act, qa, M, K, MP, GS);
@@ -609,6 +737,11 @@ cudaError_t launch_strip(const int8_t* qa, const uint16_t* sa, const int32_t* as
     a.status = reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF);
     a.slots = reinterpret_cast<unsigned long long*>(ws + WS_HEADER_BYTES);
     a.debug_partials = debug_partials;
+    a.h = fuse ? static_cast<__nv_bfloat16*>(fuse->h) : nullptr;
+    a.qa_h = fuse ? fuse->qa_h : nullptr;
+    a.sa_h = fuse ? fuse->sa_h : nullptr;
+    a.asum_h = fuse ? fuse->asum_h : nullptr;
+    a.sync = reinterpret_cast<uint32_t*>(ws + WS_FUSE_SYNC_OFF);
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)ctas, 1, 1);
@@ -620,15 +753,21 @@ cudaError_t launch_strip(const int8_t* qa, const uint16_t* sa, const int32_t* as
     attrs[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attrs;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_strip_kernel<MB, RBLK, DEBUG>, tm_act, tm_nib, tm_scale, tm_zero, a);
+    return cudaLaunchKernelEx(&cfg, gemm_strip_kernel<MB, RBLK, DEBUG, FUSE>, tm_act, tm_nib, tm_scale, tm_zero, a);
 }
 
 template <int MB, int RBLK>
 cudaError_t launch_strip_dbg(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed, void* y,
-                             int M, int N, int K, int ctas, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
+                             int M, int N, int K, int ctas, void* workspace, int32_t* debug_partials, const FuseOut* fuse,
+                             cudaStream_t stream) {
+    if (fuse) {
+        // two token blocks always run on 32-row strips (strip_plan): the other widths are not built in the fused form
+        if constexpr (MB == 2 && RBLK != 2) return cudaErrorInvalidConfiguration;
+        else return launch_strip<MB, RBLK, false, true>(qa, sa, asum, packed, nullptr, M, N, K, ctas, workspace, nullptr, fuse, stream);
+    }
     if (debug_partials)
-        return launch_strip<MB, RBLK, true>(qa, sa, asum, packed, y, M, N, K, ctas, workspace, debug_partials, stream);
-    return launch_strip<MB, RBLK, false>(qa, sa, asum, packed, y, M, N, K, ctas, workspace, nullptr, stream);
+        return launch_strip<MB, RBLK, true, false>(qa, sa, asum, packed, y, M, N, K, ctas, workspace, debug_partials, nullptr, stream);
+    return launch_strip<MB, RBLK, false, false>(qa, sa, asum, packed, y, M, N, K, ctas, workspace, nullptr, nullptr, stream);
 }
 
 }  // namespace
@@ -682,13 +821,14 @@ void strip_plan(int M, int N, int K, int* strip_rows, int* ctas) {
     if (ctas) *ctas = c;
 }
 
-cudaError_t launch_gemm_strip(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
-                              void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
-                              cudaStream_t stream) {
+namespace {
+cudaError_t strip_dispatch(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
+                           void* y, int M, int N, int K, void* workspace, int32_t* debug_partials, const FuseOut* fuse,
+                           cudaStream_t stream) {
     int R = 0, ctas = 0;
     strip_plan(M, N, K, &R, &ctas);
 #define W4A8_STRIP_CASE(MBV, RBV) \
-    return launch_strip_dbg<MBV, RBV>(qa, sa, asum, packed, y, M, N, K, ctas, workspace, debug_partials, stream)
+    return launch_strip_dbg<MBV, RBV>(qa, sa, asum, packed, y, M, N, K, ctas, workspace, debug_partials, fuse, stream)
     if (M <= 8) {
         if (R == 128) W4A8_STRIP_CASE(1, 8);
         if (R == 64) W4A8_STRIP_CASE(1, 4);
@@ -700,6 +840,22 @@ cudaError_t launch_gemm_strip(const int8_t* qa, const uint16_t* sa, const int32_
     if (R == 32) W4A8_STRIP_CASE(2, 2);
     W4A8_STRIP_CASE(2, 1);
 #undef W4A8_STRIP_CASE
+}
+}  // namespace
+
+cudaError_t launch_gemm_strip(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
+                              void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
+                              cudaStream_t stream) {
+    return strip_dispatch(qa, sa, asum, packed, y, M, N, K, workspace, debug_partials, nullptr, stream);
+}
+
+// The fused gate+up form: packed = the 2 I = N channels in runs of eight gate / eight up; outputs h [M, I] bf16 and the
+// quantised input of the down projection (codes, token scales, group sums).  I must be a multiple of 128.
+cudaError_t launch_gemm_strip_gate_up(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
+                                      int M, int N, int K, void* h, int8_t* qa_h, uint16_t* sa_h, int32_t* asum_h,
+                                      void* workspace, cudaStream_t stream) {
+    const FuseOut f = {h, qa_h, sa_h, asum_h};
+    return strip_dispatch(qa, sa, asum, packed, nullptr, M, N, K, workspace, nullptr, &f, stream);
 }
 
 }  // namespace w4a8

@@ -13,6 +13,7 @@
 // zero-point correction term) come from a 16-lane segmented shuffle: 16 chunks of 8 = one group of 128.
 #include <cuda_fp16.h>
 #include "ptx_sm100.cuh"
+#include "quant_common.cuh"
 #include "w4a8_internal.cuh"
 
 namespace w4a8 {
@@ -27,14 +28,6 @@ __device__ __forceinline__ uint32_t absmax_bits_bf16x8(const uint4& v, uint32_t 
     run = __vmaxu2(run, v.z & 0x7FFF7FFFu);
     run = __vmaxu2(run, v.w & 0x7FFF7FFFu);
     return run;
-}
-
-__device__ __forceinline__ int quant1(uint32_t bf16_hi_bits, float s) {
-    // bf16_hi_bits: the value's bits already in the upper half of a 32-bit word
-    float q = __fdiv_rn(__uint_as_float(bf16_hi_bits), s);
-    int r;
-    asm("cvt.rni.sat.s8.f32 %0, %1;" : "=r"(r) : "f"(q));   // ties to even, saturates to [-128,127]
-    return max(r, -127);
 }
 
 __device__ __forceinline__ uint2 quant8(const uint4& v, float s, int& sum) {
@@ -72,10 +65,15 @@ __device__ __forceinline__ uint32_t quant4_fast(uint32_t lo_pair, uint32_t hi_pa
 // division as the tie fallback - for many rows, where instruction issue matters; with few rows the kernel is a single
 // latency chain and the shorter code of the plain division is quicker (1.8 against 1.9 us at 8 rows, 2.0 against
 // 2.7 us at 128).
-template <int QA_THREADS, int QA_CACHE, bool FAST>
+//
+// SILU: the input row is the bf16 output of a fused gate+up projection, 2 K values in 16-byte chunks that
+// alternate between eight gate channels and the eight up channels of the same indices; the row that is quantised
+// is h = bf16(SiLU(gate) * up), K values, computed chunk by chunk as it is loaded (Sec. 3.5: the element-wise
+// step merged into its consumer) and, if h_out is given, also stored.
+template <int QA_THREADS, int QA_CACHE, bool FAST, bool SILU>
 __global__ void __launch_bounds__(QA_THREADS, QA_THREADS == 256 ? (QA_CACHE == 2 ? 8 : 5) : (QA_THREADS == 512 ? 3 : 1))
 quantize_act_kernel(const uint4* __restrict__ x, int K, uint2* __restrict__ qa,
-                    uint16_t* __restrict__ sa, int32_t* __restrict__ asum) {
+                    uint16_t* __restrict__ sa, int32_t* __restrict__ asum, uint4* __restrict__ h_out) {
     // Under programmatic dependent launch this grid may start while its predecessor still runs:
     // let the next grid start as early, and touch no memory before the predecessor is complete.
     ptx::pdl_launch_dependents();
@@ -83,8 +81,19 @@ quantize_act_kernel(const uint4* __restrict__ x, int K, uint2* __restrict__ qa,
     const int m = blockIdx.x;
     const int chunks = K >> 3;                    // 16-byte chunks per row; a multiple of 16
     const int G = K >> 7;
-    const uint4* xr = x + (size_t)m * chunks;
+    const uint4* xr = x + (size_t)m * chunks * (SILU ? 2 : 1);
     uint2* qr = qa + (size_t)m * chunks;
+    // chunk c of the row to quantise
+    auto load = [&](int c) -> uint4 {
+        if (!SILU) return __ldcg(xr + c);
+        const uint4 g = __ldcg(xr + 2 * c), u = __ldcg(xr + 2 * c + 1);
+        uint4 h;
+        h.x = silu_mul_bf16x2(g.x, u.x);
+        h.y = silu_mul_bf16x2(g.y, u.y);
+        h.z = silu_mul_bf16x2(g.z, u.z);
+        h.w = silu_mul_bf16x2(g.w, u.w);
+        return h;
+    };
     const int tid = threadIdx.x;
 
     uint4 cache[QA_CACHE];
@@ -93,12 +102,12 @@ quantize_act_kernel(const uint4* __restrict__ x, int K, uint2* __restrict__ qa,
     for (int i = 0; i < QA_CACHE; ++i) {
         int c = tid + i * QA_THREADS;
         if (c < chunks) {
-            cache[i] = __ldcg(xr + c);
+            cache[i] = load(c);
             run = absmax_bits_bf16x8(cache[i], run);
         }
     }
     for (int c = tid + QA_CACHE * QA_THREADS; c < chunks; c += QA_THREADS)
-        run = absmax_bits_bf16x8(__ldcg(xr + c), run);
+        run = absmax_bits_bf16x8(load(c), run);
 
     uint32_t mx = max(run & 0xFFFFu, run >> 16);
     mx = __reduce_max_sync(0xFFFFFFFFu, mx);
@@ -108,8 +117,7 @@ quantize_act_kernel(const uint4* __restrict__ x, int K, uint2* __restrict__ qa,
 #pragma unroll
     for (int w = 0; w < QA_THREADS / 32; ++w) mx = max(mx, warp_max[w]);
 
-    const float amax = __uint_as_float(mx << 16);
-    const __half sh = __float2half_rn(fminf(__fdiv_rn(amax, 127.0f), 65504.0f));
+    const __half sh = row_scale_from_amax_bits(mx);
     const float s = __half2float(sh);
     if (tid == 0) sa[m] = __half_as_ushort(sh);
     // the fast path needs a quotient that cannot leave [-127.1, 127.1]: not for a saturated scale
@@ -134,6 +142,7 @@ quantize_act_kernel(const uint4* __restrict__ x, int K, uint2* __restrict__ qa,
             if (worst > 0.5f - 0.0001220703125f) o = quant8(v, s, sum);      // 2^-13: a possible tie in this chunk
         }
         qr[c] = o;
+        if (SILU && h_out) h_out[(size_t)m * chunks + c] = v;
         sum += __shfl_xor_sync(seg_mask, sum, 8);
         sum += __shfl_xor_sync(seg_mask, sum, 4);
         sum += __shfl_xor_sync(seg_mask, sum, 2);
@@ -145,13 +154,15 @@ quantize_act_kernel(const uint4* __restrict__ x, int K, uint2* __restrict__ qa,
         int c = tid + i * QA_THREADS;
         if (c < chunks) emit(c, cache[i]);
     }
-    for (int c = tid + QA_CACHE * QA_THREADS; c < chunks; c += QA_THREADS) emit(c, __ldcg(xr + c));
+    for (int c = tid + QA_CACHE * QA_THREADS; c < chunks; c += QA_THREADS) emit(c, load(c));
 }
 
 }  // namespace
 
-cudaError_t launch_quantize_act(const void* x, int M, int K, int8_t* qa, uint16_t* sa, int32_t* asum,
-                                cudaStream_t stream) {
+namespace {
+template <bool SILU>
+cudaError_t launch_quantize(const void* x, int M, int K, int8_t* qa, uint16_t* sa, int32_t* asum, void* h_out,
+                            cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)M, 1, 1);
     // measured on B200 (K = 4096 and 12288): 512 threads per row are best up to 512 rows except between
@@ -166,13 +177,26 @@ cudaError_t launch_quantize_act(const void* x, int M, int K, int8_t* qa, uint16_
     cfg.numAttrs = 1;
     const uint4* xp = reinterpret_cast<const uint4*>(x);
     uint2* qp = reinterpret_cast<uint2*>(qa);
+    uint4* hp = reinterpret_cast<uint4*>(h_out);
     if (threads == 1024)
-        return cudaLaunchKernelEx(&cfg, quantize_act_kernel<1024, QA_CACHE_CHUNKS / 1024, false>, xp, K, qp, sa, asum);
+        return cudaLaunchKernelEx(&cfg, quantize_act_kernel<1024, QA_CACHE_CHUNKS / 1024, false, SILU>, xp, K, qp, sa, asum, hp);
     if (threads == 512)
-        return cudaLaunchKernelEx(&cfg, quantize_act_kernel<512, QA_CACHE_CHUNKS / 512, false>, xp, K, qp, sa, asum);
+        return cudaLaunchKernelEx(&cfg, quantize_act_kernel<512, QA_CACHE_CHUNKS / 512, false, SILU>, xp, K, qp, sa, asum, hp);
     if (K <= 256 * 2 * 8)                                    // rows of up to 4096: two chunks per thread, eight rows per SM
-        return cudaLaunchKernelEx(&cfg, quantize_act_kernel<256, 2, true>, xp, K, qp, sa, asum);
-    return cudaLaunchKernelEx(&cfg, quantize_act_kernel<256, QA_CACHE_CHUNKS / 256, true>, xp, K, qp, sa, asum);
+        return cudaLaunchKernelEx(&cfg, quantize_act_kernel<256, 2, true, SILU>, xp, K, qp, sa, asum, hp);
+    return cudaLaunchKernelEx(&cfg, quantize_act_kernel<256, QA_CACHE_CHUNKS / 256, true, SILU>, xp, K, qp, sa, asum, hp);
+}
+}  // namespace
+
+cudaError_t launch_quantize_act(const void* x, int M, int K, int8_t* qa, uint16_t* sa, int32_t* asum,
+                                cudaStream_t stream) {
+    return launch_quantize<false>(x, M, K, qa, sa, asum, nullptr, stream);
+}
+
+// y_gate_up: bf16 [M, 2 I] in the chunk-interleaved layout; quantises h = SiLU(gate) * up, [M, I]
+cudaError_t launch_silu_mul_quantize(const void* y_gate_up, int M, int I, void* h_out, int8_t* qa, uint16_t* sa,
+                                     int32_t* asum, cudaStream_t stream) {
+    return launch_quantize<true>(y_gate_up, M, I, qa, sa, asum, h_out, stream);
 }
 
 }  // namespace w4a8

@@ -44,6 +44,7 @@ constexpr int BLOB_BYTES = BLOB_ZERO_OFF + TILE_N / 2;        // 8512
 //                             (all zero between calls: the tag is what says that a word has been written)
 //   [SHARED, ...)             split-K fp32 slices  [S][M][N], or the tensor-core kernel's hand-over tiles
 constexpr int WS_STATUS_OFF = 0;
+constexpr int WS_FUSE_SYNC_OFF = 64;    // fused gate+up form: 16 per-token maxima, arrivals, departures (18 words)
 constexpr int WS_COUNTER_OFF = 256;
 constexpr int WS_HEADER_BYTES = W4A8_WORKSPACE_HEADER_BYTES;
 constexpr int MAX_N_TILES = (WS_HEADER_BYTES - WS_COUNTER_OFF) / 4;   // 960 tiles = N up to 122880
@@ -71,6 +72,10 @@ cudaError_t make_strip_weight_maps(CUtensorMap* nib, CUtensorMap* scale, CUtenso
 cudaError_t make_qa_group_map(CUtensorMap* out, const int8_t* qa, int M, int K, int box_rows, int box_groups);
 cudaError_t launch_quantize_act(const void* x, int M, int K, int8_t* qa, uint16_t* sa, int32_t* asum,
                                 cudaStream_t stream);
+// h = bf16(SiLU(gate) * up) of a chunk-interleaved gate+up output y [M, 2 I], quantised like an activation row;
+// h_out (bf16 [M, I]) may be null
+cudaError_t launch_silu_mul_quantize(const void* y_gate_up, int M, int I, void* h_out, int8_t* qa, uint16_t* sa,
+                                     int32_t* asum, cudaStream_t stream);
 cudaError_t launch_pack_weights(const uint8_t* qw, const uint16_t* scales, const uint8_t* zeros,
                                 int N, int K, void* packed, cudaStream_t stream);
 cudaError_t launch_unpack_weights(const void* packed, int N, int K, uint8_t* qw, uint16_t* scales,
@@ -90,6 +95,10 @@ void strip_plan(int M, int N, int K, int* strip_rows, int* ctas);
 cudaError_t launch_gemm_strip(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
                               void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
                               cudaStream_t stream);
+// the strip kernel with the fused SiLU * up -> requantise epilogue (one launch; needs strip_supported and I % 128 == 0)
+cudaError_t launch_gemm_strip_gate_up(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
+                                      int M, int N, int K, void* h, int8_t* qa_h, uint16_t* sa_h, int32_t* asum_h,
+                                      void* workspace, cudaStream_t stream);
 int device_sm_count();                       // SMs of the current device (cached per device)
 int cluster_num_slices(int M, int N, int K);
 cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
