@@ -425,8 +425,41 @@ def run_layer_chain(torch, B, peaks, l2_bytes, timer):
         nbytes = sum(step_bytes(M, L["N"], L["K"]) for L in layers)
         t_roof = sum(max(wl.algorithmic_ops(M, L["N"], L["K"]) / (int8_peak * 1e12),
                          step_bytes(M, L["N"], L["K"]) / (peaks["hbm_gbs"] * 1e9)) for L in layers)
-        out.append({"M": M, "us_per_layer": round(us, 2), "kernels_per_layer": 8, "tops": round(ops / us / 1e6, 1),
-                    "gbs": round(nbytes / us / 1e3, 1), "frac_measured": round(t_roof * 1e6 / us, 3)})
+        row = {"M": M, "us_per_layer": round(us, 2), "kernels_per_layer": 8, "tops": round(ops / us / 1e6, 1),
+               "gbs": round(nbytes / us / 1e3, 1), "frac_measured": round(t_roof * 1e6 / us, 3)}
+        # The same layer with the fused gate+up step: the projection's epilogue (or, above 16 tokens, the quantiser that
+        # follows it) forms SiLU(gate) * up and the down projection's quantised input, which the down projection then
+        # takes as it is - the real data dependency of a decoder layer, one kernel fewer where the fusion is one kernel.
+        # Fractions use the same roofline sum as above (the same logical work).
+        by_name = dict(zip(wl.LAYERS.keys(), layers))
+        gu, dn = by_name["gate_up"], by_name["down"]
+        I = gu["N"] // 2
+        assert dn["K"] == I
+        h_out = (torch.empty((M, I), dtype=torch.bfloat16, device="cuda"), torch.empty((M, I), dtype=torch.int8, device="cuda"),
+                 torch.empty((M,), dtype=torch.float16, device="cuda"), torch.empty((M, I // 128), dtype=torch.int32, device="cuda"))
+        form_names = {B.GATE_UP_EPILOGUE: "SiLU*up in the strip kernel's epilogue + requantise kernel",
+                      B.GATE_UP_ONE_KERNEL: "one kernel (epilogue, last CTAs stay and requantise)",
+                      B.GATE_UP_SEPARATE: "GEMM + SiLU*up quantiser"}
+        forms = [B.w4a8_gate_up_form(M, gu["N"], gu["K"])] + ([B.GATE_UP_ONE_KERNEL] if M <= 16 else [])
+        for fi, form in enumerate(forms):
+            def body_fused():
+                for _ in range(reps):
+                    for c in range(ncopies):
+                        for name in ("qkv", "o"):
+                            L = by_name[name]
+                            B.w4a8_linear(L["xm"], L["packed"][c], L["N"], L["ws"], 128, out=L["y"], scratch=L["scratch"])
+                        B.w4a8_quantize_act(gu["xm"], 128, out=gu["scratch"])
+                        B.w4a8_gate_up_silu_quantize(gu["scratch"][0], gu["scratch"][1], gu["scratch"][2], gu["packed"][c], gu["N"],
+                                                     gu["ws"], 128, form=form, y_scratch=gu["y"], out=h_out)
+                        B.w4a8_gemm(h_out[1], h_out[2], h_out[3], dn["packed"][c], dn["N"], dn["ws"], 128, out=dn["y"])
+            _, times = timer.graph_ms(body_fused, replays=5, warm=2)
+            for L in layers:
+                B.w4a8_check_status(L["ws"])
+            usf = min(times) * 1e3 / (reps * ncopies)
+            row["fused_gate_up" if fi == 0 else "fused_gate_up_one_kernel"] = {
+                "us_per_layer": round(usf, 2), "kernels_per_layer": 7 if form == B.GATE_UP_ONE_KERNEL else 8,
+                "frac_measured": round(t_roof * 1e6 / usf, 3), "form": form_names[form]}
+        out.append(row)
     del layers
     torch.cuda.empty_cache()
     return out

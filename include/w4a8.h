@@ -178,23 +178,36 @@ w4a8_status w4a8_plan(int M, int N, int K, int group, w4a8_plan_info* out);
  *   qa_h       device, int8 [M, I]; sa_h fp16 [M]; asum_h int32 [M, I / 128]
  *   I % 128 == 0, group == 128.  One kernel, one CTA per token.
  *
- * w4a8_gate_up_silu_quantize: projection and step together.  Where w4a8_gemm would take the strip kernel
- * (w4a8_gate_up_is_one_kernel returns 1: up to 8 tokens, and 9..16 on wide layers) this is ONE kernel: the
- * strip kernel's epilogue forms h from its own sums, the CTAs meet at a grid-wide barrier (bounded wait; the
- * grid is sized so that every CTA is resident), and all warps then quantise h; y is never stored.  Otherwise
- * it is w4a8_gemm into y_scratch followed by w4a8_silu_mul_quantize, with identical results.
+ * w4a8_gate_up_silu_quantize: projection and step together, in one of three forms (results identical bit for bit):
+ *   W4A8_GATE_UP_EPILOGUE    the strip kernel's epilogue forms h from its own sums, stores it and keeps each token's
+ *                            largest |h| (atomic maxima); y is never stored.  A second, small kernel (one warp per token
+ *                            and group of 128) quantises h once the maxima are final: the kernel boundary is the
+ *                            grid-wide wait.  Where the strip kernel runs (M <= 16, see w4a8_plan).
+ *   W4A8_GATE_UP_ONE_KERNEL  the same epilogue, but the requantisation stays inside the kernel: every CTA counts itself in,
+ *                            the last 128 to arrive stay, wait (bounded) until all have, and quantise.  One launch fewer;
+ *                            measured slower than the form above on B200 (the stayers' wait for the last stores of h to
+ *                            become visible costs more than a dependent launch), kept for comparison.
+ *   W4A8_GATE_UP_SEPARATE    w4a8_gemm into y_scratch, then w4a8_silu_mul_quantize.  Any M.
+ *   W4A8_GATE_UP_AUTO        EPILOGUE where w4a8_gemm would take the strip kernel, else SEPARATE (w4a8_gate_up_form says
+ *                            which, 0 for an unsupported shape).
  *   qa, sa, asum, packed_gate_up, M, N (= 2 I), K, group, workspace: as for w4a8_gemm
- *   h          device, bf16 [M, I]: output, and in the one-kernel form also the buffer through which the
- *              CTAs exchange h (required)
- *   y_scratch  device, bf16 [M, N]; needed only when w4a8_gate_up_is_one_kernel returns 0, else may be NULL
- * Errors as for w4a8_gemm, W4A8_ERR_SHAPE also for I % 128 != 0.  The one-kernel form keeps 18 words of the
- * workspace header (per-token maxima and two counters) that it leaves zero; after W4A8_ERR_TIMEOUT the
- * workspace must be initialised again before its next use.
+ *   h          device, bf16 [M, I]: output, and in the first two forms also the buffer through which h reaches the
+ *              warps that quantise it (required)
+ *   y_scratch  device, bf16 [M, N]; needed only by the SEPARATE form, else may be NULL
+ * Errors as for w4a8_gemm; W4A8_ERR_SHAPE also for I % 128 != 0, an unknown form, or a strip-kernel form where that kernel
+ * does not exist (M > 16).  The strip-kernel forms keep 18 words of the workspace header (per-token maxima and two
+ * counters) that they leave zero; after W4A8_ERR_TIMEOUT the workspace must be initialised again before its next use.
  */
+typedef enum {
+    W4A8_GATE_UP_AUTO = 0,
+    W4A8_GATE_UP_ONE_KERNEL = 1,
+    W4A8_GATE_UP_EPILOGUE = 2,
+    W4A8_GATE_UP_SEPARATE = 3
+} w4a8_gate_up_form_t;
 w4a8_status w4a8_silu_mul_quantize(const void* y_gate_up_bf16, int M, int I, int group, void* h_bf16,
                                    int8_t* qa_h, uint16_t* sa_h, int32_t* asum_h, void* stream);
-int w4a8_gate_up_is_one_kernel(int M, int N, int K, int group);
-w4a8_status w4a8_gate_up_silu_quantize(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
+int w4a8_gate_up_form(int M, int N, int K, int group);
+w4a8_status w4a8_gate_up_silu_quantize(int form, const int8_t* qa, const uint16_t* sa, const int32_t* asum,
                                        const void* packed_gate_up, int M, int N, int K, int group,
                                        void* h_bf16, int8_t* qa_h, uint16_t* sa_h, int32_t* asum_h,
                                        void* y_scratch_bf16, void* workspace, size_t workspace_bytes,

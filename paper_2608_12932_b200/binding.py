@@ -22,7 +22,7 @@ EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w
            "w4a8_pack_weights", "w4a8_unpack_weights", "w4a8_quantize_act", "w4a8_gemm", "w4a8_gemm_path",
            "w4a8_linear", "w4a8_linear_host", "w4a8_gemm_static_scratch", "w4a8_check_status", "w4a8_plan",
            "w4a8_gemm_per_channel", "w4a8_static_scratch_status", "w4a8_selftest_wait_timeout",
-           "w4a8_silu_mul_quantize", "w4a8_gate_up_is_one_kernel", "w4a8_gate_up_silu_quantize")
+           "w4a8_silu_mul_quantize", "w4a8_gate_up_form", "w4a8_gate_up_silu_quantize")
 
 _lib = None
 
@@ -66,10 +66,10 @@ def lib():
         L.w4a8_plan.argtypes = [ci, ci, ci, ci, vp]
         L.w4a8_silu_mul_quantize.restype = ci
         L.w4a8_silu_mul_quantize.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp]
-        L.w4a8_gate_up_is_one_kernel.restype = ci
-        L.w4a8_gate_up_is_one_kernel.argtypes = [ci, ci, ci, ci]
+        L.w4a8_gate_up_form.restype = ci
+        L.w4a8_gate_up_form.argtypes = [ci, ci, ci, ci]
         L.w4a8_gate_up_silu_quantize.restype = ci
-        L.w4a8_gate_up_silu_quantize.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.w4a8_gate_up_silu_quantize.argtypes = [ci, vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, sz, vp]
         L.w4a8_linear.restype = ci
         L.w4a8_linear.argtypes = [vp, vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, sz, vp]
         L.w4a8_linear_host.restype = ci
@@ -236,21 +236,27 @@ def w4a8_silu_mul_quantize(y_gate_up, group=GROUP, out=None, stream=None):
     return h, qa_h, sa_h, asum_h
 
 
-def w4a8_gate_up_is_one_kernel(M, N, K, group=GROUP):
-    return bool(lib().w4a8_gate_up_is_one_kernel(M, N, K, group))
+GATE_UP_AUTO, GATE_UP_ONE_KERNEL, GATE_UP_EPILOGUE, GATE_UP_SEPARATE = 0, 1, 2, 3
 
 
-def w4a8_gate_up_silu_quantize(qa, sa, asum, packed_gate_up, N, workspace, group=GROUP, y_scratch=None, out=None, stream=None):
-    """Fused gate+up projection, SiLU(gate) * up and the down projection's activation quantisation: one kernel where
-    w4a8_gemm would take the strip kernel, else the GEMM into y_scratch followed by w4a8_silu_mul_quantize."""
+def w4a8_gate_up_form(M, N, K, group=GROUP):
+    """The form GATE_UP_AUTO takes for this size (0 for an unsupported shape)."""
+    return int(lib().w4a8_gate_up_form(M, N, K, group))
+
+
+def w4a8_gate_up_silu_quantize(qa, sa, asum, packed_gate_up, N, workspace, group=GROUP, form=GATE_UP_AUTO, y_scratch=None,
+                               out=None, stream=None):
+    """Fused gate+up projection, SiLU(gate) * up and the down projection's activation quantisation; see the header for
+    the three forms.  Returns (h, qa_h, sa_h, asum_h)."""
     _dev(qa, torch.int8, "qa"), _dev(sa, torch.float16, "sa"), _dev(asum, torch.int32, "asum")
     _dev(packed_gate_up, torch.uint8, "packed_gate_up"), _dev(workspace, torch.uint8, "workspace")
     M, K = qa.shape
     I = N // 2
     h, qa_h, sa_h, asum_h = _h_outputs(M, I, group, qa.device, out)
-    if y_scratch is None and M > 0 and not w4a8_gate_up_is_one_kernel(M, N, K, group):
+    separate = form == GATE_UP_SEPARATE or (form == GATE_UP_AUTO and w4a8_gate_up_form(M, N, K, group) == GATE_UP_SEPARATE)
+    if y_scratch is None and M > 0 and separate:
         y_scratch = torch.empty((M, N), dtype=torch.bfloat16, device=qa.device)
-    _check(lib().w4a8_gate_up_silu_quantize(_ptr(qa), _ptr(sa), _ptr(asum), _ptr(packed_gate_up), M, N, K, group,
+    _check(lib().w4a8_gate_up_silu_quantize(form, _ptr(qa), _ptr(sa), _ptr(asum), _ptr(packed_gate_up), M, N, K, group,
                                             _ptr(h), _ptr(qa_h), _ptr(sa_h), _ptr(asum_h), _ptr(y_scratch),
                                             _ptr(workspace), workspace.numel(), _stream(stream)),
            "w4a8_gate_up_silu_quantize")

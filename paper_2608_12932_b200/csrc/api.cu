@@ -200,20 +200,25 @@ w4a8_status w4a8_silu_mul_quantize(const void* y_gate_up_bf16, int M, int I, int
                ? W4A8_OK : W4A8_ERR_CUDA;
 }
 
-int w4a8_gate_up_is_one_kernel(int M, int N, int K, int group) {
+int w4a8_gate_up_form(int M, int N, int K, int group) {
     if (!shape_ok(N, K, group) || M < 1 || (N / 2) % GROUP != 0) return 0;
-    return auto_takes_strip(M, N, K) ? 1 : 0;
+    return auto_takes_strip(M, N, K) ? W4A8_GATE_UP_EPILOGUE : W4A8_GATE_UP_SEPARATE;
 }
 
-w4a8_status w4a8_gate_up_silu_quantize(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed_gate_up,
-                                       int M, int N, int K, int group, void* h_bf16, int8_t* qa_h, uint16_t* sa_h,
-                                       int32_t* asum_h, void* y_scratch_bf16, void* workspace, size_t workspace_bytes,
-                                       void* stream) {
+w4a8_status w4a8_gate_up_silu_quantize(int form, const int8_t* qa, const uint16_t* sa, const int32_t* asum,
+                                       const void* packed_gate_up, int M, int N, int K, int group, void* h_bf16,
+                                       int8_t* qa_h, uint16_t* sa_h, int32_t* asum_h, void* y_scratch_bf16,
+                                       void* workspace, size_t workspace_bytes, void* stream) {
     if (!shape_ok(N, K, group) || M < 0 || (N / 2) % GROUP != 0) return W4A8_ERR_SHAPE;
+    if (form != W4A8_GATE_UP_AUTO && form != W4A8_GATE_UP_ONE_KERNEL && form != W4A8_GATE_UP_EPILOGUE &&
+        form != W4A8_GATE_UP_SEPARATE)
+        return W4A8_ERR_SHAPE;
     if (M == 0) return W4A8_OK;
+    if (form == W4A8_GATE_UP_AUTO) form = w4a8_gate_up_form(M, N, K, group);
+    // the two forms that live in the strip kernel's epilogue exist where that kernel does
+    if (form != W4A8_GATE_UP_SEPARATE && !strip_supported(M, N, K)) return W4A8_ERR_SHAPE;
     if (!qa || !sa || !asum || !packed_gate_up || !h_bf16 || !qa_h || !sa_h || !asum_h || !workspace) return W4A8_ERR_NULL;
-    const bool one = w4a8_gate_up_is_one_kernel(M, N, K, group) != 0;
-    if (!one && !y_scratch_bf16) return W4A8_ERR_NULL;
+    if (form == W4A8_GATE_UP_SEPARATE && !y_scratch_bf16) return W4A8_ERR_NULL;
     if (!aligned(qa, 16) || !aligned(sa, 2) || !aligned(asum, 4) || !aligned(packed_gate_up, 128) || !aligned(h_bf16, 16) ||
         !aligned(qa_h, 16) || !aligned(sa_h, 2) || !aligned(asum_h, 4) || !aligned(workspace, 256) ||
         (y_scratch_bf16 && !aligned(y_scratch_bf16, 16)))
@@ -222,8 +227,9 @@ w4a8_status w4a8_gate_up_silu_quantize(const int8_t* qa, const uint16_t* sa, con
     w4a8_status a = arch_check();
     if (a != W4A8_OK) return a;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (one)
-        return launch_gemm_strip_gate_up(qa, sa, asum, packed_gate_up, M, N, K, h_bf16, qa_h, sa_h, asum_h, workspace, st) == cudaSuccess
+    if (form != W4A8_GATE_UP_SEPARATE)
+        return launch_gemm_strip_gate_up(qa, sa, asum, packed_gate_up, M, N, K, h_bf16, qa_h, sa_h, asum_h,
+                                         form == W4A8_GATE_UP_ONE_KERNEL, workspace, st) == cudaSuccess
                    ? W4A8_OK : W4A8_ERR_CUDA;
     w4a8_status g = w4a8_gemm_path(W4A8_PATH_AUTO, qa, sa, asum, packed_gate_up, y_scratch_bf16, M, N, K, group, workspace,
                                    workspace_bytes, nullptr, stream);

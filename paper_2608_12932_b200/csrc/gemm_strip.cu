@@ -70,6 +70,7 @@ constexpr int ST_THREADS = (ST_CONSUMER_WARPS + ST_PRODUCER_WARPS + 1) * 32;
 constexpr int ST_MAX_STAGES = 8;
 constexpr int ST_W_BYTES = ST_CW == 8 ? 17408 : 26624;                         // weight part of a stage (16 KB of nibbles + scales + zero points, padded)
 constexpr int ST_SMEM_BUDGET = 112 * 1024;                // per CTA: two launches share an SM
+constexpr uint32_t ST_STAY = 128;                         // one-kernel fused form: CTAs that stay to requantise (swept 32..296 on B200)
 constexpr int ST_MAX_ASUM_WORDS = 4096;                   // group sums of all tokens kept in shared memory
 
 struct StLayout {
@@ -125,12 +126,34 @@ __device__ __forceinline__ bool st_wait(uint32_t bar, uint32_t parity, volatile 
     }
 }
 
+// h[m, 128 g .. 128 g + 127] -> codes, group sum and (for g == 0) the token's scale; one warp, four values per lane
+__device__ __forceinline__ void requant_unit(const __nv_bfloat16* h, int I, int Gh, int u, int lane, int8_t* qa_h,
+                                             uint16_t* sa_h, int32_t* asum_h, const uint32_t* sync) {
+    const int m = u / Gh, g = u - m * Gh;
+    const size_t at = (size_t)m * I + (size_t)g * GROUP + 4 * lane;
+    const uint2 hv = __ldcg(reinterpret_cast<const uint2*>(h + at));
+    const __half sh = row_scale_from_amax_bits(__ldcg(sync + m));
+    const float s = __half2float(sh);
+    int q0 = 0, q1 = 0, q2 = 0, q3 = 0;
+    if (s != 0.0f) {
+        q0 = quant1(hv.x << 16, s); q1 = quant1(hv.x & 0xFFFF0000u, s);
+        q2 = quant1(hv.y << 16, s); q3 = quant1(hv.y & 0xFFFF0000u, s);
+    }
+    *reinterpret_cast<uint32_t*>(qa_h + at) =
+        (uint32_t)(q0 & 0xFF) | ((uint32_t)(q1 & 0xFF) << 8) | ((uint32_t)(q2 & 0xFF) << 16) | ((uint32_t)q3 << 24);
+    const int sum = __reduce_add_sync(0xFFFFFFFFu, q0 + q1 + q2 + q3);
+    if (lane == 0) {
+        asum_h[(size_t)m * Gh + g] = sum;
+        if (g == 0) sa_h[m] = __half_as_ushort(sh);
+    }
+}
+
 #ifdef W4A8_TRACE
-// working builds only: time stamps of one launch's stages, [launch % 64][CTA][16] words
-__device__ unsigned long long g_strip_trace[64 * 192 * 96];
-__device__ unsigned int g_strip_trace_count[192];
-#define ST_STAMP(k) do { g_strip_trace[((size_t)(trace_launch & 63) * 192 + blockIdx.x) * 96 + (k)] = ptx::globaltimer_ns(); } while (0)
-#define ST_PUT(k, v) do { g_strip_trace[((size_t)(trace_launch & 63) * 192 + blockIdx.x) * 96 + (k)] = (unsigned long long)(v); } while (0)
+// working builds only: time stamps of one launch's stages, [launch % 64][CTA < 320][96] words
+__device__ unsigned long long g_strip_trace[64 * 320 * 96];
+__device__ unsigned int g_strip_trace_count[320];
+#define ST_STAMP(k) do { g_strip_trace[((size_t)(trace_launch & 63) * 320 + blockIdx.x) * 96 + (k)] = ptx::globaltimer_ns(); } while (0)
+#define ST_PUT(k, v) do { g_strip_trace[((size_t)(trace_launch & 63) * 320 + blockIdx.x) * 96 + (k)] = (unsigned long long)(v); } while (0)
 #define ST_CLK() clock64()
 #else
 #define ST_STAMP(k) do { } while (0)
@@ -162,11 +185,11 @@ struct StripArgs {
 // runs of eight (rows 16 b .. 16 b + 7 of the packed layer are gate channels 8 b .. 8 b + 7, rows 16 b + 8 .. 16 b + 15
 // the up channels of the same indices), so that a lane of the epilogue warp holds gate and up of one channel.  The
 // epilogue rounds both to bf16 as the plain kernel would, computes h = bf16(SiLU(gate) * up), stores h and keeps
-// the largest |h| per token; all CTAs then meet at a grid-wide barrier (every CTA of the grid is resident: the
-// launcher bounds the grid by the occupancy), after which the warps of all CTAs quantise h, one (token, group of
-// 128) per warp: codes, token scales and group sums of the down projection's input leave this kernel; y is never
-// stored.
-template <int MB, int RBLK, bool DEBUG, bool FUSE>
+// the largest |h| per token (atomic maxima in the workspace); y is never stored.  What remains is to quantise h once
+// every token's maximum is final, one (token, group of 128) per warp.  FUSE == 2: a second, small kernel does that
+// (requant_kernel below; the kernel boundary is the grid-wide wait).  FUSE == 1, the one-kernel form: every CTA
+// counts itself in; the last 128 to do so stay, wait (bounded) until the count is complete, and quantise.
+template <int MB, int RBLK, bool DEBUG, int FUSE>
 __global__ void __launch_bounds__(ST_THREADS, 2)
 gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_nib,
                   const __grid_constant__ CUtensorMap tm_scale, const __grid_constant__ CUtensorMap tm_zero,
@@ -612,62 +635,60 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
                     const int m = 8 * mb + 2 * j + t;
                     if (r == 0 && m < a.M && v != 0u) atomicMax(a.sync + m, v);
                 }
-            __threadfence();                                   // h and the maxima before the arrival
-            __syncwarp();
-            if (lane == 0) atomicAdd(a.sync + 16, 1u);
+            __syncwarp();                                      // the lanes' stores of h and maxima, then one release
+            // one-kernel form: the CTA's place in the order of arrival decides whether it stays for the requantisation
+            if (FUSE == 1 && lane == 0) {
+                uint32_t place;
+                asm volatile("atom.add.release.gpu.global.u32 %0, [%1], 1;" : "=r"(place) : "l"(a.sync + 16) : "memory");
+                *reinterpret_cast<volatile uint32_t*>(smem + L.misc_off + 4) = place;
+            }
         }
         if (lane == 0) ST_STAMP(6);
     }
     __syncwarp();
-    if (FUSE) {
-        // ---- grid-wide barrier, then the requantisation of h by all warps of all CTAs ----
+    if (FUSE == 1) {
+        // ---- the last CTAs to arrive wait for the rest and requantise h; the others leave at once ----
+        // (a CTA that leaves frees its place for the next kernel's CTAs, which start their weight stream under this
+        // kernel's tail; a stayer waits only for CTAs that run or will run whether it holds its place or not, so the
+        // grid need not be resident as a whole)
         __syncthreads();
-        if (tid == 0) {
-            uint64_t t0 = 0;
-            for (uint32_t spin = 0; !*abort_flag; ++spin) {
-                uint32_t v;
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a.sync + 16) : "memory");
-                if (v >= gridDim.x) break;
-                if ((spin & 15) == 15) {
-                    const uint64_t now = ptx::globaltimer_ns();
-                    if (t0 == 0) t0 = now;
-                    else if (now - t0 > ptx::WAIT_LIMIT_NS) { *abort_flag = 1; break; }
+        const uint32_t stay = gridDim.x < ST_STAY ? gridDim.x : ST_STAY;
+        const uint32_t place = *reinterpret_cast<volatile uint32_t*>(smem + L.misc_off + 4);
+        if (tid == 0) { ST_STAMP(7); ST_PUT(12, place); }
+        if (place >= gridDim.x - stay) {
+            const uint32_t rank = place - (gridDim.x - stay);
+            if (tid == 0) {
+                uint64_t t0 = 0;
+                for (uint32_t spin = 0; !*abort_flag; ++spin) {
+                    uint32_t v;
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a.sync + 16) : "memory");
+                    if (v >= gridDim.x) break;
+                    if ((spin & 15) == 15) {
+                        const uint64_t now = ptx::globaltimer_ns();
+                        if (t0 == 0) t0 = now;
+                        else if (now - t0 > ptx::WAIT_LIMIT_NS) { *abort_flag = 1; break; }
+                    }
                 }
-                __nanosleep(100);
-            }
-            __threadfence();
-        }
-        __syncthreads();
-        if (!*abort_flag) {
-            const int I = a.N / 2, Gh = I / GROUP;
-            constexpr int WARPS = ST_THREADS / 32;
-            for (int u = blockIdx.x * WARPS + warp; u < a.M * Gh; u += gridDim.x * WARPS) {
-                const int m = u / Gh, g = u - m * Gh;
-                const __half sh = row_scale_from_amax_bits(__ldcg(a.sync + m));
-                const float s = __half2float(sh);
-                const size_t at = (size_t)m * I + (size_t)g * GROUP + 4 * lane;
-                const uint2 hv = __ldcg(reinterpret_cast<const uint2*>(a.h + at));
-                int q0 = 0, q1 = 0, q2 = 0, q3 = 0;
-                if (s != 0.0f) {
-                    q0 = quant1(hv.x << 16, s); q1 = quant1(hv.x & 0xFFFF0000u, s);
-                    q2 = quant1(hv.y << 16, s); q3 = quant1(hv.y & 0xFFFF0000u, s);
-                }
-                *reinterpret_cast<uint32_t*>(a.qa_h + at) =
-                    (uint32_t)(q0 & 0xFF) | ((uint32_t)(q1 & 0xFF) << 8) | ((uint32_t)(q2 & 0xFF) << 16) | ((uint32_t)q3 << 24);
-                const int sum = __reduce_add_sync(0xFFFFFFFFu, q0 + q1 + q2 + q3);
-                if (lane == 0) {
-                    a.asum_h[(size_t)m * Gh + g] = sum;
-                    if (g == 0) a.sa_h[m] = __half_as_ushort(sh);
-                }
-            }
-        }
-        __syncthreads();
-        // the last CTA to leave puts the words back to zero for the next call
-        if (tid == 0) {
-            const uint32_t old = atomicAdd(a.sync + 17, 1u);
-            if (old == gridDim.x - 1) {
-                for (int i = 0; i < 18; ++i) a.sync[i] = 0u;
                 __threadfence();
+                ST_STAMP(8);
+            }
+            __syncthreads();
+            if (!*abort_flag) {
+                const int I = a.N / 2, Gh = I / GROUP;
+                constexpr int WARPS = ST_THREADS / 32;
+                for (int u = (int)rank * WARPS + warp; u < a.M * Gh; u += (int)stay * WARPS)
+                    requant_unit(a.h, I, Gh, u, lane, a.qa_h, a.sa_h, a.asum_h, a.sync);
+            }
+            __syncthreads();
+            // the last stayer to leave puts the words back to zero for the next call
+            if (tid == 0) ST_STAMP(9);
+            if (tid == 0) {
+                const uint32_t old = atomicAdd(a.sync + 17, 1u);
+                if (old == stay - 1) {
+                    for (int i = 0; i < 18; ++i) a.sync[i] = 0u;
+                    __threadfence();
+                }
+                ST_STAMP(13);
             }
         }
     }
@@ -680,14 +701,35 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
     }
 }
 
+// The quantisation of h after the gate+up kernel in its two-kernel form: one (token, group of 128) per warp, the
+// token's scale from its final maximum.  The last CTA to finish puts the maxima back to zero for the next call.
+__global__ void __launch_bounds__(256) requant_kernel(const __nv_bfloat16* __restrict__ h, int M, int I, int8_t* __restrict__ qa_h,
+                                                      uint16_t* __restrict__ sa_h, int32_t* __restrict__ asum_h, uint32_t* sync) {
+    ptx::pdl_launch_dependents();
+    ptx::pdl_wait();
+    const int Gh = I / GROUP, lane = threadIdx.x & 31;
+    const int u = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (u < M * Gh) requant_unit(h, I, Gh, u, lane, qa_h, sa_h, asum_h, sync);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const uint32_t old = atomicAdd(sync + 17, 1u);
+        if (old == gridDim.x - 1) {
+            for (int i = 0; i < 18; ++i) sync[i] = 0u;
+            __threadfence();
+        }
+    }
+}
+
 struct FuseOut {
     void* h;
     int8_t* qa_h;
     uint16_t* sa_h;
     int32_t* asum_h;
+    bool one_kernel;
 };
 
-template <int MB, int RBLK, bool DEBUG, bool FUSE>
+template <int MB, int RBLK, bool DEBUG, int FUSE>
 cudaError_t launch_strip(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed, void* y,
                          int M, int N, int K, int ctas, void* workspace, int32_t* debug_partials, const FuseOut* fuse,
                          cudaStream_t stream) {
@@ -713,8 +755,8 @@ cudaError_t launch_strip(const int8_t* qa, const uint16_t* sa, const int32_t* as
         resident[dev] = per_sm * device_sm_count();
         attr_done[dev] = true;
     }
-    if (FUSE) {
-        // the grid-wide barrier needs every CTA resident at the same time
+    if (FUSE == 1) {
+        // keep the grid within what is resident at once: the stayers then never wait for a CTA that has yet to start
         if (resident[dev] < 1) return cudaErrorInvalidConfiguration;
         if (ctas > resident[dev]) ctas = resident[dev];
     }
@@ -753,7 +795,14 @@ cudaError_t launch_strip(const int8_t* qa, const uint16_t* sa, const int32_t* as
     attrs[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attrs;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_strip_kernel<MB, RBLK, DEBUG, FUSE>, tm_act, tm_nib, tm_scale, tm_zero, a);
+    e = cudaLaunchKernelEx(&cfg, gemm_strip_kernel<MB, RBLK, DEBUG, FUSE>, tm_act, tm_nib, tm_scale, tm_zero, a);
+    if (e != cudaSuccess || FUSE != 2) return e;
+    // two-kernel form: the requantisation once every maximum is final
+    const int units = M * (N / 2 / GROUP);
+    cfg.gridDim = dim3((unsigned)((units + 7) / 8), 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    return cudaLaunchKernelEx(&cfg, requant_kernel, (const __nv_bfloat16*)a.h, M, N / 2, a.qa_h, a.sa_h, a.asum_h, a.sync);
 }
 
 template <int MB, int RBLK>
@@ -763,19 +812,22 @@ cudaError_t launch_strip_dbg(const int8_t* qa, const uint16_t* sa, const int32_t
     if (fuse) {
         // two token blocks always run on 32-row strips (strip_plan): the other widths are not built in the fused form
         if constexpr (MB == 2 && RBLK != 2) return cudaErrorInvalidConfiguration;
-        else return launch_strip<MB, RBLK, false, true>(qa, sa, asum, packed, nullptr, M, N, K, ctas, workspace, nullptr, fuse, stream);
+        else if (fuse->one_kernel)
+            return launch_strip<MB, RBLK, false, 1>(qa, sa, asum, packed, nullptr, M, N, K, ctas, workspace, nullptr, fuse, stream);
+        else
+            return launch_strip<MB, RBLK, false, 2>(qa, sa, asum, packed, nullptr, M, N, K, ctas, workspace, nullptr, fuse, stream);
     }
     if (debug_partials)
-        return launch_strip<MB, RBLK, true, false>(qa, sa, asum, packed, y, M, N, K, ctas, workspace, debug_partials, nullptr, stream);
-    return launch_strip<MB, RBLK, false, false>(qa, sa, asum, packed, y, M, N, K, ctas, workspace, nullptr, nullptr, stream);
+        return launch_strip<MB, RBLK, true, 0>(qa, sa, asum, packed, y, M, N, K, ctas, workspace, debug_partials, nullptr, stream);
+    return launch_strip<MB, RBLK, false, 0>(qa, sa, asum, packed, y, M, N, K, ctas, workspace, nullptr, nullptr, stream);
 }
 
 }  // namespace
 
 #ifdef W4A8_TRACE
 extern "C" int w4a8_strip_trace_read(unsigned long long* host_out, unsigned int* host_counts) {
-    if (cudaMemcpyFromSymbol(host_out, g_strip_trace, sizeof(unsigned long long) * 64 * 192 * 96) != cudaSuccess) return 1;
-    if (cudaMemcpyFromSymbol(host_counts, g_strip_trace_count, sizeof(unsigned int) * 192) != cudaSuccess) return 2;
+    if (cudaMemcpyFromSymbol(host_out, g_strip_trace, sizeof(unsigned long long) * 64 * 320 * 96) != cudaSuccess) return 1;
+    if (cudaMemcpyFromSymbol(host_counts, g_strip_trace_count, sizeof(unsigned int) * 320) != cudaSuccess) return 2;
     return 0;
 }
 #endif
@@ -853,8 +905,8 @@ cudaError_t launch_gemm_strip(const int8_t* qa, const uint16_t* sa, const int32_
 // quantised input of the down projection (codes, token scales, group sums).  I must be a multiple of 128.
 cudaError_t launch_gemm_strip_gate_up(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
                                       int M, int N, int K, void* h, int8_t* qa_h, uint16_t* sa_h, int32_t* asum_h,
-                                      void* workspace, cudaStream_t stream) {
-    const FuseOut f = {h, qa_h, sa_h, asum_h};
+                                      bool one_kernel, void* workspace, cudaStream_t stream) {
+    const FuseOut f = {h, qa_h, sa_h, asum_h, one_kernel};
     return strip_dispatch(qa, sa, asum, packed, nullptr, M, N, K, workspace, nullptr, &f, stream);
 }
 

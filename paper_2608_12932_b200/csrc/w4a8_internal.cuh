@@ -95,10 +95,11 @@ void strip_plan(int M, int N, int K, int* strip_rows, int* ctas);
 cudaError_t launch_gemm_strip(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
                               void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
                               cudaStream_t stream);
-// the strip kernel with the fused SiLU * up -> requantise epilogue (one launch; needs strip_supported and I % 128 == 0)
+// the strip kernel with the SiLU * up epilogue, then the requantisation of h: by a second small kernel, or
+// (one_kernel) by the CTAs that arrive last (needs strip_supported and I % 128 == 0)
 cudaError_t launch_gemm_strip_gate_up(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
                                       int M, int N, int K, void* h, int8_t* qa_h, uint16_t* sa_h, int32_t* asum_h,
-                                      void* workspace, cudaStream_t stream);
+                                      bool one_kernel, void* workspace, cudaStream_t stream);
 int device_sm_count();                       // SMs of the current device (cached per device)
 int cluster_num_slices(int M, int N, int K);
 cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,

@@ -102,52 +102,61 @@ SHAPES = [(1, 256, 128), (4, 512, 256), (8, 1024, 384), (8, 4096, 12288), (3, 38
 
 
 @pytest.mark.parametrize("M,K,I", SHAPES)
-def test_gate_up_fused_against_oracle_and_two_kernel_form(M, K, I):
+def test_gate_up_forms_against_oracle_and_one_another(M, K, I):
     N = 2 * I
     c, packed = fused_layer(K, I, 900 + M, M)
     ws = B.new_workspace(max(M, 16), N, K)
     x = t_u16(c["x"], torch.bfloat16)
     qa, sa, asum = B.w4a8_quantize_act(x)
-    one = B.w4a8_gate_up_is_one_kernel(M, N, K)
-    assert one == (B.w4a8_plan(M, N, K)["family"] == B.PATH_STRIP)
-    outs = []
-    for rep in range(3):                                       # the workspace words must come back to zero each time
-        h, qa_h, sa_h, asum_h = B.w4a8_gate_up_silu_quantize(qa, sa, asum, packed, N, ws)
-        torch.cuda.synchronize()
-        B.w4a8_check_status(ws)
-        outs.append((bits(h), qa_h.cpu().numpy(), bits(sa_h), asum_h.cpu().numpy()))
-    for o in outs[1:]:
-        assert all(np.array_equal(a, b) for a, b in zip(o, outs[0]))
-    hb = outs[0][0]
-    # the projection by itself, same kernel family, and the step applied to its output: the same bits
-    y = B.w4a8_gemm(qa, sa, asum, packed, N, ws)
-    B.w4a8_check_status(ws)
-    h2, qa2, sa2, asum2 = B.w4a8_silu_mul_quantize(y)
-    torch.cuda.synchronize()
-    assert np.array_equal(bits(h2), hb) and np.array_equal(qa2.cpu().numpy(), outs[0][1])
-    assert np.array_equal(bits(sa2), outs[0][2]) and np.array_equal(asum2.cpu().numpy(), outs[0][3])
-    # h against the oracle on the kernel's own y; codes against the oracle's quantiser on the kernel's h
-    gate_b, up_b = split_fused(bits(y), I)
-    check_h(hb, gate_b, up_b)
-    check_codes(hb, qa_h, sa_h, asum_h)
-    # the whole chain against the oracle on the unfused matrices: rows 0..I-1 gate, I..2I-1 up
-    ref = cfast.w4a8_linear(c["x"], c["qw"], c["sw"], c["z"], 128)["ref"]
+    auto = B.w4a8_gate_up_form(M, N, K)
+    strip = B.w4a8_plan(M, N, K)["family"] == B.PATH_STRIP
+    assert auto == (B.GATE_UP_EPILOGUE if strip else B.GATE_UP_SEPARATE)
+    forms = [B.GATE_UP_AUTO, B.GATE_UP_SEPARATE] + ([B.GATE_UP_EPILOGUE, B.GATE_UP_ONE_KERNEL] if M <= 16 else [])
+    # Forms that multiply in the same GEMM kernel must agree bit for bit: the two epilogue forms always run the strip
+    # kernel, AUTO and SEPARATE run whatever w4a8_gemm takes for the shape.
+    groups = {}
+    for form in forms:
+        in_strip = form in (B.GATE_UP_EPILOGUE, B.GATE_UP_ONE_KERNEL) or strip
+        for rep in range(3):                                   # the workspace words must come back to zero each time
+            h, qa_h, sa_h, asum_h = B.w4a8_gate_up_silu_quantize(qa, sa, asum, packed, N, ws, form=form)
+            torch.cuda.synchronize()
+            B.w4a8_check_status(ws)
+            groups.setdefault(in_strip, []).append((form, bits(h), qa_h.cpu().numpy(), bits(sa_h), asum_h.cpu().numpy()))
+    ref = cfast.w4a8_linear(c["x"], c["qw"], c["sw"], c["z"], 128)["ref"]      # unfused matrices: rows 0..I-1 gate, I..2I-1 up
     h_ref, band = chain_band(ref, I)
-    err = np.abs(onp.bf16_bits_to_f64(hb) - h_ref)
-    assert np.all(err <= band), f"worst err/band {float((err / band).max()):.3f}"
-    # and the down projection's operands work as such: the scale reproduces h within half a step
-    sa_f = onp.fp16_bits_to_f64(outs[0][2])
-    assert np.all(np.abs(onp.bf16_bits_to_f64(hb) - sa_f[:, None] * outs[0][1]) <= sa_f[:, None] / 2 + 1e-12)
+    for in_strip, outs in groups.items():
+        first = outs[0]
+        for o in outs[1:]:
+            assert all(np.array_equal(a, b) for a, b in zip(o[1:], first[1:])), f"forms {first[0]} and {o[0]} differ"
+        hb, qa_hb, sa_hb, asum_hb = first[1:]
+        # the projection by itself in the same kernel family, and the step applied to its output: the same bits
+        y = B.w4a8_gemm(qa, sa, asum, packed, N, ws, path=B.PATH_STRIP if in_strip else B.PATH_AUTO)
+        B.w4a8_check_status(ws)
+        h2, qa2, sa2, asum2 = B.w4a8_silu_mul_quantize(y)
+        torch.cuda.synchronize()
+        assert np.array_equal(bits(h2), hb) and np.array_equal(qa2.cpu().numpy(), qa_hb)
+        assert np.array_equal(bits(sa2), sa_hb) and np.array_equal(asum2.cpu().numpy(), asum_hb)
+        # h against the oracle on the kernel's own y; codes against the oracle's quantiser on the kernel's h
+        gate_b, up_b = split_fused(bits(y), I)
+        check_h(hb, gate_b, up_b)
+        qa_o, sa_o, asum_o = onp.quantize_act(hb, 128)
+        assert np.array_equal(qa_hb, qa_o) and np.array_equal(sa_hb, sa_o) and np.array_equal(asum_hb, asum_o)
+        # the whole chain against the oracle's chain
+        err = np.abs(onp.bf16_bits_to_f64(hb) - h_ref)
+        assert np.all(err <= band), f"worst err/band {float((err / band).max()):.3f}"
+        # and the down projection's operands work as such: the scale reproduces h within half a step
+        sa_f = onp.fp16_bits_to_f64(sa_hb)
+        assert np.all(np.abs(onp.bf16_bits_to_f64(hb) - sa_f[:, None] * qa_hb) <= sa_f[:, None] / 2 + 1e-12)
 
 
-def test_one_kernel_form_covers_the_small_m_shapes():
-    assert B.w4a8_gate_up_is_one_kernel(8, 24576, 4096)
-    assert B.w4a8_gate_up_is_one_kernel(16, 24576, 4096)
-    assert not B.w4a8_gate_up_is_one_kernel(64, 24576, 4096)
-    assert not B.w4a8_gate_up_is_one_kernel(8, 24576 + 128, 4096)      # I not a multiple of 128
+def test_form_chosen_for_the_layer_shapes():
+    assert B.w4a8_gate_up_form(8, 24576, 4096) == B.GATE_UP_EPILOGUE
+    assert B.w4a8_gate_up_form(16, 24576, 4096) == B.GATE_UP_EPILOGUE
+    assert B.w4a8_gate_up_form(64, 24576, 4096) == B.GATE_UP_SEPARATE
+    assert B.w4a8_gate_up_form(8, 24576 + 128, 4096) == 0               # I not a multiple of 128
 
 
-def test_two_kernel_form_needs_its_scratch_and_shapes_are_checked():
+def test_separate_form_needs_its_scratch_and_shapes_are_checked():
     M, K, I = 64, 256, 256
     c, packed = fused_layer(K, I, 5, M)
     ws = B.new_workspace(M, 2 * I, K)
@@ -157,9 +166,14 @@ def test_two_kernel_form_needs_its_scratch_and_shapes_are_checked():
     sa_h = torch.empty((M,), dtype=torch.float16, device="cuda")
     asum_h = torch.empty((M, I // 128), dtype=torch.int32, device="cuda")
     L = B.lib()
-    args = [B._ptr(qa), B._ptr(sa), B._ptr(asum), B._ptr(packed), M, 2 * I, K, 128, B._ptr(h), B._ptr(qa_h), B._ptr(sa_h),
-            B._ptr(asum_h), None, B._ptr(ws), ws.numel(), None]
+    args = [B.GATE_UP_AUTO, B._ptr(qa), B._ptr(sa), B._ptr(asum), B._ptr(packed), M, 2 * I, K, 128, B._ptr(h), B._ptr(qa_h),
+            B._ptr(sa_h), B._ptr(asum_h), None, B._ptr(ws), ws.numel(), None]
     assert L.w4a8_gate_up_silu_quantize(*args) == B.ERR_NULL
-    args[5] = 2 * I + 128                                       # N / 2 not a multiple of 128
+    args[0] = B.GATE_UP_ONE_KERNEL                              # no strip kernel at 64 tokens
+    assert L.w4a8_gate_up_silu_quantize(*args) == B.ERR_SHAPE
+    args[0] = 7
+    assert L.w4a8_gate_up_silu_quantize(*args) == B.ERR_SHAPE
+    args[0] = B.GATE_UP_AUTO
+    args[6] = 2 * I + 128                                       # N / 2 not a multiple of 128
     assert L.w4a8_gate_up_silu_quantize(*args) == B.ERR_SHAPE
     torch.cuda.synchronize()
