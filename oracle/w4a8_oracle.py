@@ -138,6 +138,40 @@ def silu_mul_quantize(y_gate_bits, y_up_bits, group):
     return dict(h=h, h_bits=h_bits, qa=qa, sa=sa_bits, asum=asum)
 
 
+# ---- the weight-only variant the paper argues against (Sec. 3.4, first paragraph) ------------------
+def dequantize_weights(qw, sw_bits, z, group):
+    """w[n,k] = s_w[g(k),n] * (q_w[n,k] - z[g(k),n]) in fp64 (exact: an 11-bit by a 5-bit factor), and its bf16 rounding.
+    Returns (w fp64 [N,K], bf16 bits [N,K])."""
+    qw = np.asarray(qw).astype(np.int64)
+    N, K = qw.shape
+    sw = fp16_bits_to_f64(sw_bits)
+    zz = np.asarray(z).astype(np.int64)
+    w = np.empty((N, K), dtype=np.float64)
+    for g in range(K // group):
+        ks = slice(g * group, (g + 1) * group)
+        w[:, ks] = sw[g][:, None] * (qw[:, ks] - zz[g][:, None]).astype(np.float64)
+    return w, f64_to_bf16_bits(w)
+
+
+def w4a16_linear(x_bits, qw, sw_bits, z, group):
+    """W4A16: the same 4-bit weights against UNQUANTISED bf16 activations (the AWQ-style weight-only scheme the
+    paper contrasts W4A8 with: it shrinks the weights, which helps the memory-bound decode, and leaves the
+    multiplications in 16-bit floating point).  ref[m,n] = sum_g s_w[g,n] * sum_{k in g} x[m,k] (q_w[n,k] - z[g,n])
+    in fp64, group by group.  Returns ref [M,N] fp64; a kernel's bf16 result is judged with the band below."""
+    x = bf16_bits_to_f64(x_bits)
+    qw = np.asarray(qw).astype(np.int64)
+    zz = np.asarray(z).astype(np.int64)
+    sw = fp16_bits_to_f64(sw_bits)
+    M, K = x.shape
+    N = qw.shape[0]
+    ref = np.zeros((M, N), dtype=np.float64)
+    for g in range(K // group):
+        ks = slice(g * group, (g + 1) * group)
+        P = x[:, ks] @ (qw[:, ks] - zz[g][:, None]).astype(np.float64).T          # [M,N]
+        ref += sw[g][None, :] * P
+    return ref
+
+
 # ---- acceptance band for a bf16 result ------------------------------------------------
 def tolerance(ref):
     """Per-element bound 2^-7 |ref| + 1e-3 rms(ref), rms over the whole [M,N] result."""

@@ -455,3 +455,62 @@ def test_silu_mul_quantize_is_the_quantiser_on_h():
     # codes: h / sa = 126.98, -51.02, -125.16, 0, 18.03, -0.156 -> 127, -51, -125, 0, 18, 0
     assert q["qa"][0].tolist() == [127, -51, -125, 0, 18, 0, 0, 0]
     assert q["asum"][0].tolist() == [127 - 51 - 125 + 18]
+
+
+# ---- W4A16: the weight-only variant (Sec. 3.4, first paragraph) -------------------------------------
+def test_w4a16_worked_example(golden):
+    g8 = golden("worked_example_w4a8.txt")
+    g16 = golden("worked_example_w4a16.txt")
+    group = g8["group"][0]
+    x = bits_bf16([g8["x"]])
+    qw = np.array([g8["qw_row0"], g8["qw_row1"]], dtype=np.uint8)
+    z = np.array([g8["z_row0"], g8["z_row1"]], dtype=np.uint8).T.copy()
+    sw = bits_fp16(np.array([g8["sw_row0"], g8["sw_row1"]]).T.copy())
+    ref = onp.w4a16_linear(x, qw, sw, z, group)
+    assert ref[0].tolist() == g16["ref"]
+    assert onp.f64_to_bf16_bits(ref)[0].tolist() == g16["y_bf16_bits"]
+    w, w_bits = onp.dequantize_weights(qw, sw, z, group)
+    assert w[0].tolist() == g16["w_row0"] and w[1].tolist() == g16["w_row1"]
+    assert np.array_equal(onp.bf16_bits_to_f64(w_bits), w)                     # these happen to be bf16 numbers
+
+
+def test_w4a16_brute_force_on_exact_rationals():
+    rng = np.random.default_rng(21)
+    for M, N, K, group in ((2, 3, 8, 4), (1, 2, 12, 4), (3, 1, 16, 8)):
+        c = wl.random_codes(rng, M, N, K, group)
+        ref = onp.w4a16_linear(c["x"], c["qw"], c["sw"], c["z"], group)
+        x = [[Fraction(float(v)) for v in row] for row in onp.bf16_bits_to_f64(c["x"])]
+        sw = [[Fraction(float(v)) for v in row] for row in onp.fp16_bits_to_f64(c["sw"])]
+        for m in range(M):
+            for n in range(N):
+                y = sum(x[m][k] * sw[k // group][n] * (int(c["qw"][n, k]) - int(c["z"][k // group, n])) for k in range(K))
+                assert abs(float(y) - ref[m, n]) <= 1e-13 * max(1.0, abs(float(y)))
+
+
+def test_w4a16_reduces_to_dgemm_and_meets_w4a8_where_quantisation_is_exact():
+    rng = np.random.default_rng(22)
+    M, N, K, group = 5, 24, 256, 128
+    c = wl.random_codes(rng, M, N, K, group)
+    ref = onp.w4a16_linear(c["x"], c["qw"], c["sw"], c["z"], group)
+    w, w_bits = onp.dequantize_weights(c["qw"], c["sw"], c["z"], group)
+    assert np.allclose(ref, onp.bf16_bits_to_f64(c["x"]) @ w.T, rtol=1e-12, atol=1e-12)            # library dgemm
+    # dequantised weights: one exact product per element, and the bf16 rounding is the pinned one
+    assert np.array_equal(w_bits, onp.f64_to_bf16_bits(w))
+    assert np.abs(onp.bf16_bits_to_f64(w_bits) - w).max() <= 2.0 ** -8 * np.abs(w).max()
+    # Activations that the W4A8 quantiser reproduces exactly (integers -127..127 times a power of two, the largest
+    # magnitude 127 so that the scale is that power of two): both schemes then compute the same sum.
+    q = rng.integers(-127, 128, size=(M, K))
+    q[:, 0] = 127
+    xq = wl.f32_to_bf16_bits((q * 2.0 ** -5).astype(np.float32))
+    r8 = onp.w4a8_linear(xq, c["qw"], c["sw"], c["z"], group)
+    assert np.array_equal(r8["qa"], q.astype(np.int8)) and np.all(onp.fp16_bits_to_f64(r8["sa"]) == 2.0 ** -5)
+    r16 = onp.w4a16_linear(xq, c["qw"], c["sw"], c["z"], group)
+    assert np.allclose(r16, r8["ref"], rtol=1e-13, atol=0)
+    # and in general the two differ by no more than the activation quantisation allows: |x - sa qa| <= sa / 2
+    r8 = onp.w4a8_linear(c["x"], c["qw"], c["sw"], c["z"], group)
+    sa = onp.fp16_bits_to_f64(r8["sa"])
+    assert np.all(np.abs(ref - r8["ref"]) <= (sa[:, None] / 2) * np.abs(w).sum(axis=1)[None, :] + 1e-9)
+    # linear in x (exactly, for a power of two), columns independent
+    x2 = wl.f32_to_bf16_bits((onp.bf16_bits_to_f64(c["x"]) * 4.0).astype(np.float32))
+    assert np.array_equal(onp.w4a16_linear(x2, c["qw"], c["sw"], c["z"], group), 4.0 * ref)
+    assert np.array_equal(onp.w4a16_linear(c["x"], c["qw"][5:9], c["sw"][:, 5:9], c["z"][:, 5:9], group), ref[:, 5:9])
