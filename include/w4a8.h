@@ -214,6 +214,24 @@ w4a8_status w4a8_gate_up_silu_quantize(int form, const int8_t* qa, const uint16_
                                        void* stream);
 
 /*
+ * The weight-only variant the paper contrasts W4A8 with (Sec. 3.4, first paragraph: 4-bit weights with 16-bit
+ * activations shrink what the memory-bound decode must load, and leave the arithmetic of the compute-bound
+ * prefill in 16-bit floating point).  Same packed weights, activations NOT quantised:
+ *   y[m,n] = bf16( sum_groups s_w[g,n] * sum_{k in g} x[m,k] (q_w[n,k] - z[g,n]) )
+ * w4a8_a16_gemm: the decode form, 1 <= M <= 16 (W4A8_ERR_SHAPE above): the strip kernel's streaming skeleton with
+ * bf16 tensor-core MMAs; a code minus its zero point is an exact bf16 integer, products are exact in fp32, a group's
+ * sum is scaled in fp32: no weight is rounded before it is multiplied.  Judged with the same band as w4a8_gemm
+ * against the fp64 definition.
+ *   x        device, bf16 [M,K] row-major, 16-byte aligned
+ *   packed_w, y, N, K, group, workspace: as for w4a8_gemm
+ * w4a8_dequantize_weights: the prefill form's first half: W[n,k] = bf16_rne(s_w (q_w - z)), row-major [N,K] bf16
+ * (device, 16-byte aligned), for a library bf16 GEMM; one rounding per weight, bit-exact against the definition.
+ */
+w4a8_status w4a8_a16_gemm(const void* x_bf16, const void* packed_w, void* y_bf16, int M, int N, int K, int group,
+                          void* workspace, size_t workspace_bytes, void* stream);
+w4a8_status w4a8_dequantize_weights(const void* packed_w, int N, int K, int group, void* w_bf16, void* stream);
+
+/*
  * Variant for weights whose scale does not change along K (per-channel scales: the paper does not
  * give its group size, Sec. 3.4; this is the coarsest choice, group 128 the library's default).
  * Same packed format and the same per-group zero points; the caller guarantees that the scales of

@@ -22,7 +22,8 @@ EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w
            "w4a8_pack_weights", "w4a8_unpack_weights", "w4a8_quantize_act", "w4a8_gemm", "w4a8_gemm_path",
            "w4a8_linear", "w4a8_linear_host", "w4a8_gemm_static_scratch", "w4a8_check_status", "w4a8_plan",
            "w4a8_gemm_per_channel", "w4a8_static_scratch_status", "w4a8_selftest_wait_timeout",
-           "w4a8_silu_mul_quantize", "w4a8_gate_up_form", "w4a8_gate_up_silu_quantize")
+           "w4a8_silu_mul_quantize", "w4a8_gate_up_form", "w4a8_gate_up_silu_quantize", "w4a8_a16_gemm",
+           "w4a8_dequantize_weights")
 
 _lib = None
 
@@ -66,6 +67,10 @@ def lib():
         L.w4a8_plan.argtypes = [ci, ci, ci, ci, vp]
         L.w4a8_silu_mul_quantize.restype = ci
         L.w4a8_silu_mul_quantize.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp]
+        L.w4a8_a16_gemm.restype = ci
+        L.w4a8_a16_gemm.argtypes = [vp, vp, vp, ci, ci, ci, ci, vp, sz, vp]
+        L.w4a8_dequantize_weights.restype = ci
+        L.w4a8_dequantize_weights.argtypes = [vp, ci, ci, ci, vp, vp]
         L.w4a8_gate_up_form.restype = ci
         L.w4a8_gate_up_form.argtypes = [ci, ci, ci, ci]
         L.w4a8_gate_up_silu_quantize.restype = ci
@@ -261,6 +266,30 @@ def w4a8_gate_up_silu_quantize(qa, sa, asum, packed_gate_up, N, workspace, group
                                             _ptr(workspace), workspace.numel(), _stream(stream)),
            "w4a8_gate_up_silu_quantize")
     return h, qa_h, sa_h, asum_h
+
+
+def w4a8_a16_gemm(x, packed_w, N, workspace, group=GROUP, out=None, stream=None):
+    """W4A16: y bf16 [M,N] from bf16 activations x [M,K] (M <= 16) and a packed layer."""
+    _dev(x, torch.bfloat16, "x"), _dev(packed_w, torch.uint8, "packed_w"), _dev(workspace, torch.uint8, "workspace")
+    M, K = x.shape
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+    else:
+        _dev(out, torch.bfloat16, "out")
+    _check(lib().w4a8_a16_gemm(_ptr(x), _ptr(packed_w), _ptr(out), M, N, K, group, _ptr(workspace), workspace.numel(),
+                               _stream(stream)), "w4a8_a16_gemm")
+    return out
+
+
+def w4a8_dequantize_weights(packed_w, N, K, group=GROUP, out=None, stream=None):
+    """Packed layer -> bf16 [N,K] weights s_w (q_w - z)."""
+    _dev(packed_w, torch.uint8, "packed_w")
+    if out is None:
+        out = torch.empty((N, K), dtype=torch.bfloat16, device=packed_w.device)
+    else:
+        _dev(out, torch.bfloat16, "out")
+    _check(lib().w4a8_dequantize_weights(_ptr(packed_w), N, K, group, _ptr(out), _stream(stream)), "w4a8_dequantize_weights")
+    return out
 
 
 class PlanInfo(ctypes.Structure):

@@ -237,6 +237,29 @@ w4a8_status w4a8_gate_up_silu_quantize(int form, const int8_t* qa, const uint16_
     return launch_silu_mul_quantize(y_scratch_bf16, M, N / 2, h_bf16, qa_h, sa_h, asum_h, st) == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
 
+w4a8_status w4a8_a16_gemm(const void* x_bf16, const void* packed_w, void* y_bf16, int M, int N, int K, int group,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+    if (!shape_ok(N, K, group) || M < 0) return W4A8_ERR_SHAPE;
+    if (M > 0 && !a16_supported(M, N, K)) return W4A8_ERR_SHAPE;
+    if (M == 0) return W4A8_OK;
+    if (!x_bf16 || !packed_w || !y_bf16 || !workspace) return W4A8_ERR_NULL;
+    if (!aligned(x_bf16, 16) || !aligned(packed_w, 128) || !aligned(y_bf16, 16) || !aligned(workspace, 256)) return W4A8_ERR_ALIGN;
+    if (workspace_bytes < w4a8_workspace_bytes(M, N, K, group)) return W4A8_ERR_WORKSPACE;
+    w4a8_status a = arch_check();
+    if (a != W4A8_OK) return a;
+    return launch_gemm_strip_a16(x_bf16, packed_w, y_bf16, M, N, K, workspace, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+w4a8_status w4a8_dequantize_weights(const void* packed_w, int N, int K, int group, void* w_bf16, void* stream) {
+    if (!shape_ok(N, K, group)) return W4A8_ERR_SHAPE;
+    if (!packed_w || !w_bf16) return W4A8_ERR_NULL;
+    if (!aligned(packed_w, 128) || !aligned(w_bf16, 16)) return W4A8_ERR_ALIGN;
+    w4a8_status a = arch_check();
+    if (a != W4A8_OK) return a;
+    return launch_dequantize_weights(packed_w, N, K, w_bf16, static_cast<cudaStream_t>(stream)) == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
 w4a8_status w4a8_gemm_per_channel(const int8_t* qa, const uint16_t* sa, const void* packed_w, void* y_bf16,
                                   int M, int N, int K, int group, void* workspace, size_t workspace_bytes,
                                   int32_t* debug_sums, void* stream) {

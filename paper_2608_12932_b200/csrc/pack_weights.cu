@@ -1,6 +1,8 @@
 // Offline weight packer and its inverse (Sec. 3.4: weights are quantised to 4 bits offline).
 // A pure permutation of codes, scales and zero points into the blob layout described in
 // w4a8_internal.cuh; one CTA per blob (128 output channels x one group of 128 k).
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include "w4a8_internal.cuh"
 
 namespace w4a8 {
@@ -58,7 +60,43 @@ unpack_weights_kernel(const uint8_t* __restrict__ packed, int N, int K, uint8_t*
     }
 }
 
+// Dequantised weights for the weight-only (W4A16) form of a large-M product: W[n,k] = bf16(s_w (q_w - z)), row-major
+// [N,K].  One CTA per blob, one thread per row: 64 packed bytes -> 128 bf16 (the product of an fp16 scale and an
+// integer of magnitude <= 15 is exact in fp32, so there is one rounding).
+__global__ void __launch_bounds__(TILE_N)
+dequantize_weights_kernel(const uint8_t* __restrict__ packed, int N, int K, __nv_bfloat16* __restrict__ W) {
+    const int G = K / GROUP;
+    const int ntile = blockIdx.x / G, g = blockIdx.x % G;
+    const uint8_t* blob = packed + (size_t)blockIdx.x * BLOB_BYTES;
+    const int r = threadIdx.x;
+    const float s = __half2float(reinterpret_cast<const __half*>(blob + BLOB_SCALE_OFF)[r]);
+    const int z = (blob[BLOB_ZERO_OFF + (r >> 1)] >> ((r & 1) * 4)) & 0xF;
+    __nv_bfloat16* dst = W + (size_t)(ntile * TILE_N + r) * K + g * GROUP;
+    for (int p = 0; p < 4; ++p) {
+        const uint4 c = *reinterpret_cast<const uint4*>(blob + r * 64 + blob_chunk_pos(r, p) * 16);
+        const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+        __align__(16) __nv_bfloat16 out[32];
+        for (int q = 0; q < 4; ++q) {
+            const int k0 = blob_word_k(q);                          // inside the chunk: 0, 4, 16, 20
+            for (int b = 0; b < 4; ++b) {
+                out[k0 + b] = __float2bfloat16_rn(s * (float)((int)((w[q] >> (8 * b)) & 0xF) - z));
+                out[k0 + 8 + b] = __float2bfloat16_rn(s * (float)((int)((w[q] >> (8 * b + 4)) & 0xF) - z));
+            }
+        }
+        uint4* d4 = reinterpret_cast<uint4*>(dst + 32 * p);
+        const uint4* o4 = reinterpret_cast<const uint4*>(out);
+        d4[0] = o4[0]; d4[1] = o4[1]; d4[2] = o4[2]; d4[3] = o4[3];
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_dequantize_weights(const void* packed, int N, int K, void* W_bf16, cudaStream_t stream) {
+    int blobs = (N / TILE_N) * (K / GROUP);
+    dequantize_weights_kernel<<<blobs, TILE_N, 0, stream>>>(static_cast<const uint8_t*>(packed), N, K,
+                                                            static_cast<__nv_bfloat16*>(W_bf16));
+    return cudaGetLastError();
+}
 
 cudaError_t launch_pack_weights(const uint8_t* qw, const uint16_t* scales, const uint8_t* zeros,
                                 int N, int K, void* packed, cudaStream_t stream) {

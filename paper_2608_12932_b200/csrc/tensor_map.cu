@@ -139,6 +139,27 @@ cudaError_t make_qa_group_map(CUtensorMap* out, const int8_t* qa, int M, int K, 
     return cudaSuccess;
 }
 
+// 3-D view of bf16 activations x[M,K] as (64 elements = 128 bytes, M tokens, K / 64 half-groups): a box of box_rows
+// tokens x box_halves half-groups lands as [half-group][token][128 B] (128-byte swizzle, zeros past M and K).
+cudaError_t make_x_half_group_map(CUtensorMap* out, const void* x, int M, int K, int box_rows, int box_halves) {
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return cudaErrorNotSupported;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const MapKey k = {x, 5, M, K, box_rows * 256 + box_halves, dev};
+    if (map_cache().find(k, out)) return cudaSuccess;
+    const cuuint64_t dims[3] = {64, (cuuint64_t)M, (cuuint64_t)(K / 64)};
+    const cuuint64_t strides[2] = {(cuuint64_t)K * 2, 128};
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_halves};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    if (encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+    map_cache().put(k, out);
+    return cudaSuccess;
+}
+
 cudaError_t make_qa_tensor_map(CUtensorMap* out, const int8_t* qa, int M, int K, int box_rows) {
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;

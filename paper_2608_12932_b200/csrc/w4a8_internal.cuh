@@ -95,6 +95,13 @@ void strip_plan(int M, int N, int K, int* strip_rows, int* ctas);
 cudaError_t launch_gemm_strip(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
                               void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
                               cudaStream_t stream);
+// W4A16 (bf16 activations against the same packed weights), up to STRIP_MAX_M tokens
+bool a16_supported(int M, int N, int K);
+void a16_plan(int M, int N, int K, int* strip_rows, int* ctas);
+cudaError_t launch_gemm_strip_a16(const void* x, const void* packed, void* y, int M, int N, int K, void* workspace,
+                                  cudaStream_t stream);
+cudaError_t launch_dequantize_weights(const void* packed, int N, int K, void* W_bf16, cudaStream_t stream);
+cudaError_t make_x_half_group_map(CUtensorMap* out, const void* x, int M, int K, int box_rows, int box_halves);
 // the strip kernel with the SiLU * up epilogue, then the requantisation of h: by a second small kernel, or
 // (one_kernel) by the CTAs that arrive last (needs strip_supported and I % 128 == 0)
 cudaError_t launch_gemm_strip_gate_up(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
