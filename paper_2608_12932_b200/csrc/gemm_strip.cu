@@ -168,6 +168,10 @@ struct StripArgs {
     __nv_bfloat16* y;
     int M, N, K;
     int stages;              // ring length
+    int pre;                 // ring slots whose weights are requested before griddepcontrol.wait (the rest: L2 prefetch).
+                             // The whole ring: fewer (1..3 slots, so that the first activation tile would not queue behind
+                             // them) changed nothing on the wide layers and cost 2 to 19 % on the narrow ones - the first
+                             // tile takes 1.5-2 us under the weight stream however little this CTA has in flight.
     int sps;                 // stages per strip = ceil(G / GS)
     int total_stages;        // strips x sps
     uint32_t* status;
@@ -273,7 +277,7 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
     const bool producer = pw >= 0 && pw < ST_PRODUCER_WARPS;
     if (producer && lane == 0) {
         // weights do not depend on the previous kernel: start their stream at once
-        const int first = n < stages ? n : stages;
+        const int first = n < a.pre ? n : a.pre;
         for (int i = pw; i < first; i += ST_PRODUCER_WARPS) load_weights(lo + i, i);
         // what the ring cannot hold is asked into L2 meanwhile, so that HBM keeps streaming under the previous
         // kernel and the ring refills from L2 (a third of the latency) once this one runs
@@ -309,6 +313,8 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
                     if (use > 0) {
                         if (!st_wait(bar_base + 8 * (ST_MAX_STAGES + s), (uint32_t)((use - 1) & 1), abort_flag)) { go = false; break; }
                         load_weights(t, s);
+                    } else if (s >= a.pre) {
+                        load_weights(t, s);                                   // ring slots not filled before the wait
                     }
                     if (i < 40) ST_STAMP(56 + i);
                     ptx::mbar_arrive_expect_tx(bar, ACT_BYTES);           // the weight bytes are announced by load_weights
@@ -774,6 +780,10 @@ cudaError_t launch_strip(const int8_t* qa, const uint16_t* sa, const int32_t* as
     a.y = static_cast<__nv_bfloat16*>(y);
     a.M = M; a.N = N; a.K = K;
     a.stages = stages;
+    a.pre = stages;
+#ifdef W4A8_TUNING
+    if (const char* e = getenv("W4A8_STRIP_PRE")) { const int v = atoi(e); if (v >= 1 && v < stages) a.pre = v; }
+#endif
     a.sps = (G + GS - 1) / GS;
     a.total_stages = (N / R) * a.sps;
     a.status = reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF);
