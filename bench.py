@@ -768,7 +768,7 @@ def run_shape(args):
 # captures summarised under profiles/ (gemm_strip_qkv_M8.md, gemm_cluster_qkv_M8.md)
 QUANTIZE_TRAFFIC_BYTES_PER_LAUNCH = 8410624      # ncu, quantize_act at 1024 x 4096 (profiles/quantize_act_M1024_K4096.md)
 TRAFFIC_BYTES_PER_LAUNCH = {"gemm_strip_kernel": 13148416, "gemm_cluster_kernel": 13144832}
-E2E_DEPTH = int(os.environ.get("W4A8_E2E_DEPTH", "4"))          # host requests in flight in the end-to-end measurement
+E2E_DEPTH = int(os.environ.get("W4A8_E2E_DEPTH", "8"))          # host requests in flight in the end-to-end measurement
 
 
 def main():
