@@ -114,6 +114,22 @@ def w4a8_linear(x_bits, qw, sw_bits, z, group):
     return dict(qa=qa, sa=sa_bits, asum=asum, D=D, ref=ref)
 
 
+# ---- a projection whose output is added to the residual stream (Sec. 3.5, "Kernel Fusion") ----
+def w4a8_linear_residual(x_bits, qw, sw_bits, z, group, residual_bits):
+    """ref[m,n] = s_a[m] sum_g s_w[g,n] D[m,g,n] + r[m,n]: the O and down projections of a decoder layer feed
+    the residual stream, and Sec. 3.5 merges such element-wise steps into their neighbours.  r is bf16 (bit
+    patterns); the sum is formed in fp64 and rounded once by whoever stores it.  Returns dict(lin, ref): the
+    projection alone and the sum (a kernel's band is taken on `lin`, see residual_tolerance)."""
+    lin = w4a8_linear(x_bits, qw, sw_bits, z, group)["ref"]
+    return dict(lin=lin, ref=lin + bf16_bits_to_f64(residual_bits))
+
+
+def residual_tolerance(lin, ref):
+    """Band for a kernel that adds the residual before its one rounding: the projection's own band (its error does
+    not shrink when the sum cancels) plus half a bf16 step of the sum."""
+    return tolerance(lin) + 2.0 ** -8 * np.abs(ref)
+
+
 # ---- the step after the fused gate+up projection (Sec. 3.5, "Kernel Fusion") -----------------
 def silu_mul(y_gate_bits, y_up_bits):
     """h[m,c] = bf16_rne( SiLU(gate[m,c]) * up[m,c] ),  SiLU(v) = v / (1 + exp(-v)),  in fp64.

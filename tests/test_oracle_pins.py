@@ -514,3 +514,33 @@ def test_w4a16_reduces_to_dgemm_and_meets_w4a8_where_quantisation_is_exact():
     x2 = wl.f32_to_bf16_bits((onp.bf16_bits_to_f64(c["x"]) * 4.0).astype(np.float32))
     assert np.array_equal(onp.w4a16_linear(x2, c["qw"], c["sw"], c["z"], group), 4.0 * ref)
     assert np.array_equal(onp.w4a16_linear(c["x"], c["qw"][5:9], c["sw"][:, 5:9], c["z"][:, 5:9], group), ref[:, 5:9])
+
+
+# ---- projection + residual (Sec. 3.5) ----------------------------------------------------------------
+def test_residual_add_worked_example_and_special_cases(golden):
+    g = golden("worked_example_w4a8.txt")
+    group = g["group"][0]
+    x = bits_bf16([g["x"]])
+    qw = np.array([g["qw_row0"], g["qw_row1"]], dtype=np.uint8)
+    z = np.array([g["z_row0"], g["z_row1"]], dtype=np.uint8).T.copy()
+    sw = bits_fp16(np.array([g["sw_row0"], g["sw_row1"]]).T.copy())
+    # by hand: -9.8419189453125 + 10 = 0.1580810546875 ; 1.1042633056640625 + (-1.125) = -0.0207366943359375
+    r = onp.w4a8_linear_residual(x, qw, sw, z, group, bits_bf16([[10.0, -1.125]]))
+    assert r["lin"][0].tolist() == g["ref"]
+    assert r["ref"][0].tolist() == [0.1580810546875, -0.0207366943359375]
+    # rounded once: 0.15808... = 1.2646484375 * 2^-3 -> mantissa 0.2646484375 * 128 = 33.875 -> 34 -> 0x3E22;
+    # 0.02073669... = 1.3271484375 * 2^-6 -> 41.875 -> 42 -> 0xBCAA   (rounding the projection first would give
+    # bf16(-9.8125 + 10) = 0.1875 = 0x3E40: the two orders differ, and the definition is the single rounding)
+    assert onp.f64_to_bf16_bits(r["ref"])[0].tolist() == [0x3E22, 0xBCAA]
+    # zero residual: the projection; codes equal to zero points: the residual itself, bit for bit
+    rng = np.random.default_rng(31)
+    c = wl.random_codes(rng, 3, 8, 256)
+    rb = wl.f32_to_bf16_bits(rng.standard_normal((3, 8)).astype(np.float32))
+    r0 = onp.w4a8_linear_residual(c["x"], c["qw"], c["sw"], c["z"], 128, np.zeros((3, 8), dtype=np.uint16))
+    assert np.array_equal(r0["ref"], onp.w4a8_linear(c["x"], c["qw"], c["sw"], c["z"], 128)["ref"])
+    qz = np.repeat(c["z"].T, 128, axis=1).astype(np.uint8)
+    rz = onp.w4a8_linear_residual(c["x"], qz, c["sw"], c["z"], 128, rb)
+    assert np.array_equal(onp.f64_to_bf16_bits(rz["ref"]), rb)
+    # the band never falls below the projection's own
+    rr = onp.w4a8_linear_residual(c["x"], c["qw"], c["sw"], c["z"], 128, rb)
+    assert np.all(onp.residual_tolerance(rr["lin"], rr["ref"]) >= onp.tolerance(rr["lin"]))
