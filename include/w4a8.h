@@ -155,6 +155,22 @@ typedef struct {
 w4a8_status w4a8_plan(int M, int N, int K, int group, w4a8_plan_info* out);
 
 /*
+ * w4a8_gemm with the residual stream added in its epilogue (Sec. 3.5, "Kernel Fusion": element-wise steps are
+ * merged into their neighbours; the O and down projections of a decoder layer feed the residual stream):
+ *   y[m,n] = bf16_rne( sa[m] * sum_groups sw[g,n] * D[m,g,n] + r[m,n] )      one rounding, the sum in fp32
+ *   residual  device, bf16 [M,N] row-major, 16-byte aligned; may be the same buffer as y (every element is read by
+ *             the thread or warp that then overwrites it)
+ *   path      W4A8_PATH_AUTO in production; the strip, cluster split-K and tensor-core families have the epilogue,
+ *             W4A8_PATH_SPLITK_WORKSPACE does not (W4A8_ERR_SHAPE)
+ * Other arguments, alignment, workspace and errors as for w4a8_gemm.  Judged against the fp64 sum with the
+ * projection's band plus half a bf16 step of the sum.
+ */
+w4a8_status w4a8_gemm_residual(w4a8_path path, const int8_t* qa, const uint16_t* sa, const int32_t* asum,
+                               const void* packed_w, const void* residual_bf16, void* y_bf16,
+                               int M, int N, int K, int group,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The step after the fused gate+up projection (Sec. 3.5, "Kernel Fusion": gate and up are one GEMM, and
  * the element-wise operations that follow are merged into their neighbours): from the projection's
  * output to the quantised input of the down projection, h never making a round trip as a separate pass.

@@ -23,7 +23,7 @@ EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w
            "w4a8_linear", "w4a8_linear_host", "w4a8_gemm_static_scratch", "w4a8_check_status", "w4a8_plan",
            "w4a8_gemm_per_channel", "w4a8_static_scratch_status", "w4a8_selftest_wait_timeout",
            "w4a8_silu_mul_quantize", "w4a8_gate_up_form", "w4a8_gate_up_silu_quantize", "w4a8_a16_gemm",
-           "w4a8_dequantize_weights")
+           "w4a8_dequantize_weights", "w4a8_gemm_residual")
 
 _lib = None
 
@@ -67,6 +67,8 @@ def lib():
         L.w4a8_plan.argtypes = [ci, ci, ci, ci, vp]
         L.w4a8_silu_mul_quantize.restype = ci
         L.w4a8_silu_mul_quantize.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp]
+        L.w4a8_gemm_residual.restype = ci
+        L.w4a8_gemm_residual.argtypes = [ci, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp]
         L.w4a8_a16_gemm.restype = ci
         L.w4a8_a16_gemm.argtypes = [vp, vp, vp, ci, ci, ci, ci, vp, sz, vp]
         L.w4a8_dequantize_weights.restype = ci
@@ -266,6 +268,20 @@ def w4a8_gate_up_silu_quantize(qa, sa, asum, packed_gate_up, N, workspace, group
                                             _ptr(workspace), workspace.numel(), _stream(stream)),
            "w4a8_gate_up_silu_quantize")
     return h, qa_h, sa_h, asum_h
+
+
+def w4a8_gemm_residual(qa, sa, asum, packed_w, residual, N, workspace, group=GROUP, out=None, path=PATH_AUTO, stream=None):
+    """y = bf16(linear + residual), one rounding; out may be the residual tensor itself."""
+    _dev(qa, torch.int8, "qa"), _dev(sa, torch.float16, "sa"), _dev(asum, torch.int32, "asum")
+    _dev(packed_w, torch.uint8, "packed_w"), _dev(workspace, torch.uint8, "workspace"), _dev(residual, torch.bfloat16, "residual")
+    M, K = qa.shape
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=qa.device)
+    else:
+        _dev(out, torch.bfloat16, "out")
+    _check(lib().w4a8_gemm_residual(path, _ptr(qa), _ptr(sa), _ptr(asum), _ptr(packed_w), _ptr(residual), _ptr(out), M, N, K, group,
+                                    _ptr(workspace), workspace.numel(), _stream(stream)), "w4a8_gemm_residual")
+    return out
 
 
 def w4a8_a16_gemm(x, packed_w, N, workspace, group=GROUP, out=None, stream=None):

@@ -149,12 +149,12 @@ w4a8_status w4a8_quantize_act(const void* x_bf16, int M, int K, int group,
                ? W4A8_OK : W4A8_ERR_CUDA;
 }
 
-w4a8_status w4a8_gemm_path(w4a8_path path,
-                           const int8_t* qa, const uint16_t* sa, const int32_t* asum,
-                           const void* packed_w, void* y_bf16,
-                           int M, int N, int K, int group,
-                           void* workspace, size_t workspace_bytes,
-                           int32_t* debug_partials, void* stream) {
+static w4a8_status gemm_impl(w4a8_path path,
+                             const int8_t* qa, const uint16_t* sa, const int32_t* asum,
+                             const void* packed_w, void* y_bf16, const void* residual,
+                             int M, int N, int K, int group,
+                             void* workspace, size_t workspace_bytes,
+                             int32_t* debug_partials, void* stream) {
     if (!shape_ok(N, K, group) || M < 0) return W4A8_ERR_SHAPE;
     if (path != W4A8_PATH_AUTO && path != W4A8_PATH_SPLITK && path != W4A8_PATH_TCGEN05 &&
         path != W4A8_PATH_SPLITK_WORKSPACE && path != W4A8_PATH_STRIP)
@@ -167,8 +167,9 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
     // workspace variant of the split-K kernel stores element by element
     if (!aligned(qa, 16) || !aligned(sa, 2) || !aligned(asum, 4) || !aligned(packed_w, 128) ||
         !aligned(y_bf16, path == W4A8_PATH_SPLITK_WORKSPACE ? 2 : 16) || !aligned(workspace, 256) ||
-        (debug_partials && !aligned(debug_partials, 4)))
+        (debug_partials && !aligned(debug_partials, 4)) || (residual && !aligned(residual, 16)))
         return W4A8_ERR_ALIGN;
+    if (residual && path == W4A8_PATH_SPLITK_WORKSPACE) return W4A8_ERR_SHAPE;     // that variant has no residual epilogue
     if (workspace_bytes < w4a8_workspace_bytes(M, N, K, group)) return W4A8_ERR_WORKSPACE;
     w4a8_status a = arch_check();
     if (a != W4A8_OK) return a;
@@ -178,12 +179,28 @@ w4a8_status w4a8_gemm_path(w4a8_path path,
         e = launch_gemm_splitk(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace,
                                reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + WS_SHARED_OFF), debug_partials, st);
     else if (path == W4A8_PATH_STRIP || (path == W4A8_PATH_AUTO && auto_takes_strip(M, N, K)))
-        e = launch_gemm_strip(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
+        e = launch_gemm_strip(qa, sa, asum, packed_w, y_bf16, residual, M, N, K, workspace, debug_partials, st);
     else if (path == W4A8_PATH_SPLITK || (path == W4A8_PATH_AUTO && !small_m_prefers_tcgen05(M, N, K, device_sm_count())))
-        e = launch_gemm_cluster(qa, sa, asum, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
+        e = launch_gemm_cluster(qa, sa, asum, packed_w, y_bf16, residual, M, N, K, workspace, debug_partials, st);
     else
-        e = launch_gemm_tcgen05(qa, sa, packed_w, y_bf16, M, N, K, workspace, debug_partials, st);
+        e = launch_gemm_tcgen05(qa, sa, packed_w, y_bf16, residual, M, N, K, workspace, debug_partials, st);
     return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+w4a8_status w4a8_gemm_path(w4a8_path path,
+                           const int8_t* qa, const uint16_t* sa, const int32_t* asum,
+                           const void* packed_w, void* y_bf16,
+                           int M, int N, int K, int group,
+                           void* workspace, size_t workspace_bytes,
+                           int32_t* debug_partials, void* stream) {
+    return gemm_impl(path, qa, sa, asum, packed_w, y_bf16, nullptr, M, N, K, group, workspace, workspace_bytes, debug_partials, stream);
+}
+
+w4a8_status w4a8_gemm_residual(w4a8_path path, const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed_w,
+                               const void* residual_bf16, void* y_bf16, int M, int N, int K, int group,
+                               void* workspace, size_t workspace_bytes, void* stream) {
+    if (M > 0 && !residual_bf16) return W4A8_ERR_NULL;
+    return gemm_impl(path, qa, sa, asum, packed_w, y_bf16, residual_bf16, M, N, K, group, workspace, workspace_bytes, nullptr, stream);
 }
 
 w4a8_status w4a8_silu_mul_quantize(const void* y_gate_up_bf16, int M, int I, int group, void* h_bf16,

@@ -76,7 +76,7 @@ template <int MB, int MINB, int RB>
 __global__ void __launch_bounds__(CL_THREADS, MINB)
 gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t* __restrict__ sa,
                     const int32_t* __restrict__ asum, const uint8_t* __restrict__ packed,
-                    __nv_bfloat16* __restrict__ y, int M, int N, int K, int S, int ng_max, int stages,
+                    __nv_bfloat16* y, const __nv_bfloat16* residual, int M, int N, int K, int S, int ng_max, int stages,
                     uint32_t* __restrict__ status, int32_t* __restrict__ debug_partials) {
     ptx::pdl_launch_dependents();
     ptx::cluster_arrive_relaxed();     // "this CTA runs": peers wait for it before they write into it
@@ -296,7 +296,12 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
     const int cnt4 = (T4 - lo4) < chunk4 ? (T4 - lo4) : chunk4;       // may be <= 0 for the last ranks
     // the token scale of this thread's first output piece: loaded now, needed after the barrier
     float t_first = 0.0f;
-    if (tid < cnt4) t_first = __half2float(__ushort_as_half(__ldcg(sa + ((lo4 + tid) >> 5))));
+    uint2 r_first = make_uint2(0u, 0u);
+    if (tid < cnt4) {
+        t_first = __half2float(__ushort_as_half(__ldcg(sa + ((lo4 + tid) >> 5))));
+        if (residual)
+            r_first = __ldcg(reinterpret_cast<const uint2*>(residual + (size_t)((lo4 + tid) >> 5) * N + (size_t)ntile * TILE_N + ((lo4 + tid) & 31) * 4));
+    }
     __syncthreads();           // the CTA's partial sums are complete in shared memory
     const float4* part4 = reinterpret_cast<const float4*>(smem + L.set_off);
     auto piece = [&](int q) {
@@ -335,8 +340,18 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
             }
             const int m = (lo4 + i) >> 5, nn = ((lo4 + i) & 31) * 4;
             const float t = (i == tid) ? t_first : __half2float(__ushort_as_half(__ldcg(sa + m)));
-            __nv_bfloat162 o01 = __floats2bfloat162_rn(acc.x * t, acc.y * t);
-            __nv_bfloat162 o23 = __floats2bfloat162_rn(acc.z * t, acc.w * t);
+            float r0 = 0.0f, r1 = 0.0f, r2 = 0.0f, r3 = 0.0f;
+            if (residual) {
+                // the projection's output joins the residual stream: added in fp32 before the one rounding (y may be
+                // the residual buffer itself: this thread reads the four values it then overwrites)
+                const uint2 rv = (i == tid) ? r_first : __ldcg(reinterpret_cast<const uint2*>(residual + (size_t)m * N + (size_t)ntile * TILE_N + nn));
+                r0 = __uint_as_float(rv.x << 16); r1 = __uint_as_float(rv.x & 0xFFFF0000u);
+                r2 = __uint_as_float(rv.y << 16); r3 = __uint_as_float(rv.y & 0xFFFF0000u);
+            }
+            float v0 = acc.x * t, v1 = acc.y * t, v2 = acc.z * t, v3 = acc.w * t;
+            if (residual) { v0 += r0; v1 += r1; v2 += r2; v3 += r3; }
+            __nv_bfloat162 o01 = __floats2bfloat162_rn(v0, v1);
+            __nv_bfloat162 o23 = __floats2bfloat162_rn(v2, v3);
             uint2 o;
             o.x = *reinterpret_cast<uint32_t*>(&o01);
             o.y = *reinterpret_cast<uint32_t*>(&o23);
@@ -346,7 +361,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmap_qa, const uint16_t*
 }
 
 template <int MB, int MINB, int RB>
-cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed, void* y,
+cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed, void* y, const void* residual,
                       int M, int N, int K, int S, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
     const int G = K / GROUP;
     const int ng_max = (G + S - 1) / S;
@@ -404,7 +419,7 @@ cudaError_t launch_mb(const int8_t* qa, const uint16_t* sa, const int32_t* asum,
     cfg.numAttrs = 3;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     return cudaLaunchKernelEx(&cfg, gemm_cluster_kernel<MB, MINB, RB>, tmap, sa, asum, static_cast<const uint8_t*>(packed),
-                              static_cast<__nv_bfloat16*>(y), M, N, K, S, ng_max, stages,
+                              static_cast<__nv_bfloat16*>(y), static_cast<const __nv_bfloat16*>(residual), M, N, K, S, ng_max, stages,
                               reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF), debug_partials);
 }
 }  // namespace
@@ -429,7 +444,7 @@ int cluster_num_slices(int M, int N, int K) {
 }
 
 cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
-                                void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
+                                void* y, const void* residual, int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream) {
     const int S = cluster_num_slices(M, N, K);
     if (M <= 8) {
@@ -437,16 +452,16 @@ cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int3
         // long enough to give every set at least two groups: more groups in flight per CTA and the
         // activation fragments are loaded once for both blocks.
         const int ng_max = (K / GROUP + S - 1) / S;
-        if (ng_max >= 8) return launch_mb<1, 2, 2>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
-        return launch_mb<1, 2, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+        if (ng_max >= 8) return launch_mb<1, 2, 2>(qa, sa, asum, packed, y, residual, M, N, K, S, workspace, debug_partials, stream);
+        return launch_mb<1, 2, 1>(qa, sa, asum, packed, y, residual, M, N, K, S, workspace, debug_partials, stream);
     }
     if (M <= 16) {
         if ((N / TILE_N) * S > device_sm_count())
-            return launch_mb<2, 2, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
-        return launch_mb<2, 1, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+            return launch_mb<2, 2, 1>(qa, sa, asum, packed, y, residual, M, N, K, S, workspace, debug_partials, stream);
+        return launch_mb<2, 1, 1>(qa, sa, asum, packed, y, residual, M, N, K, S, workspace, debug_partials, stream);
     }
-    if (M <= 32) return launch_mb<4, 1, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
-    return launch_mb<8, 1, 1>(qa, sa, asum, packed, y, M, N, K, S, workspace, debug_partials, stream);
+    if (M <= 32) return launch_mb<4, 1, 1>(qa, sa, asum, packed, y, residual, M, N, K, S, workspace, debug_partials, stream);
+    return launch_mb<8, 1, 1>(qa, sa, asum, packed, y, residual, M, N, K, S, workspace, debug_partials, stream);
 }
 
 }  // namespace w4a8

@@ -77,7 +77,7 @@ struct StLayout {
     int ring_off, bar_off, asum_off, sa_off, part_off, take_off, ystage_off, misc_off, total;
 };
 __host__ __device__ constexpr int st_stage_bytes(int mb, int rblk) { return ST_W_BYTES + (ST_UNITS / rblk) * 8 * mb * GROUP; }
-__host__ __device__ inline StLayout st_layout(int mb, int rblk, int stages, int G) {
+__host__ __device__ inline StLayout st_layout(int mb, int rblk, int stages, int G, bool fp32_stage = false) {
     const int mp = 8 * mb;
     StLayout L;
     L.ring_off = 0;                                         // stages x (weights, then GS activation tiles), 1024-aligned
@@ -87,7 +87,8 @@ __host__ __device__ inline StLayout st_layout(int mb, int rblk, int stages, int 
     L.part_off = (L.sa_off + mp * 4 + 15) & ~15;            // token scales as fp32
     L.take_off = L.part_off + ST_CONSUMER_WARPS * (rblk >= 2 ? 2 : 1) * mb * 32 * 16;   // one float4 per consumer lane, row block and token block
     L.ystage_off = L.take_off + rblk * mb * 32 * 16;        // the neighbour's sums of a shared strip
-    L.misc_off = L.ystage_off + mp * (32 * rblk + 16);      // a strip's bf16 outputs, [token][channel], rows padded by 16 B
+    // a strip's outputs, [token][channel], rows padded by 16 B: bf16, or fp32 when a residual is added at the store
+    L.misc_off = L.ystage_off + mp * ((fp32_stage ? 64 : 32) * rblk + 16);
     L.total = L.misc_off + 16;
     return L;
 }
@@ -177,6 +178,7 @@ struct StripArgs {
     uint32_t* status;
     unsigned long long* slots;   // one strip of tagged fp32 sums per CTA (STRIP_SLOT_BYTES each), zero between calls
     int32_t* debug_partials;
+    const __nv_bfloat16* residual;   // null, or bf16 [M,N] added to the projection before the one rounding (may be y)
     // fused form only (gate+up projection -> SiLU * up -> requantise): N = 2 I
     __nv_bfloat16* h;        // [M, I] bf16, written before and read after the grid-wide barrier
     int8_t* qa_h;            // [M, I]
@@ -193,6 +195,8 @@ struct StripArgs {
 // every token's maximum is final, one (token, group of 128) per warp.  FUSE == 2: a second, small kernel does that
 // (requant_kernel below; the kernel boundary is the grid-wide wait).  FUSE == 1, the one-kernel form: every CTA
 // counts itself in; the last 128 to do so stay, wait (bounded) until the count is complete, and quantise.
+// FUSE == 3 is unrelated to gate+up: the plain projection with a residual added at the store (fp32 staging, the
+// residual's 16-byte pieces requested before the wait for the consumers), for the O and down projections.
 template <int MB, int RBLK, bool DEBUG, int FUSE>
 __global__ void __launch_bounds__(ST_THREADS, 2)
 gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_nib,
@@ -224,7 +228,8 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
     uint8_t* smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
     const int G = a.K / GROUP;
     const int stages = a.stages, sps = a.sps;
-    const StLayout L = st_layout(MB, RBLK, stages, G);
+    constexpr bool SILU = FUSE == 1 || FUSE == 2;          // gate+up epilogue; FUSE == 3: residual epilogue
+    const StLayout L = st_layout(MB, RBLK, stages, G, FUSE == 3);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     // this CTA's contiguous range of stages, [lo, hi), and the strips it touches
@@ -517,6 +522,7 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
         ulonglong2* theirs = reinterpret_cast<ulonglong2*>(reinterpret_cast<uint8_t*>(a.slots) + (size_t)(blockIdx.x + 1) * SLOT);
         constexpr unsigned long long TAG = 1ull << 32;
         constexpr int HPITCH = R + 16;                            // fused form: bytes per token row of the staged h (R / 2 channels)
+        constexpr int FPITCH = 4 * R + 16;                        // with a residual: bytes per token row of the staged fp32 outputs
         uint32_t hmax[MB][2];                                     // fused form: largest |h| (bf16 bits) of this lane's tokens
 #pragma unroll
         for (int mb = 0; mb < MB; ++mb) hmax[mb][0] = hmax[mb][1] = 0u;
@@ -557,6 +563,20 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
                 if (!ok) break;
                 __syncwarp();
             }
+            // a residual joins at the store: its 16-byte pieces, in the layout of the final stores, are asked for now and
+            // have arrived by the time the consumers are done with the strip
+            constexpr int RES_CHUNKS = (MP * (R / 8) + 31) / 32;
+            uint4 rv[RES_CHUNKS];
+            constexpr bool with_res = FUSE == 3;
+            if (with_res && has_start) {
+#pragma unroll
+                for (int k = 0; k < RES_CHUNKS; ++k) {
+                    const int c = lane + 32 * k, m = c / (R / 8), col = c - m * (R / 8);
+                    rv[k] = make_uint4(0u, 0u, 0u, 0u);
+                    if (c < a.M * (R / 8))
+                        rv[k] = __ldcg(reinterpret_cast<const uint4*>(a.residual + (size_t)m * a.N + (size_t)strip * R + col * 8));
+                }
+            }
             ok = st_wait(part_full, (uint32_t)(q & 1), abort_flag);
             if (!ok) break;
             if (lane == 0 && q == nseg - 1) ST_STAMP(5);
@@ -585,10 +605,19 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
                 // bf16 outputs into the staging rows: token 8 mb + 2 j (and the next one), channels rb 16 + r and + 8
                 const int m0 = 8 * mb + 2 * j;
                 const float t0 = sa_s[m0], t1 = sa_s[m0 + 1];
+                if (with_res) {
+                    // fp32 staging: the rounding comes after the residual has been added
+                    const uint32_t fo = ystage + m0 * FPITCH + (rb * 16 + r) * 4;
+                    asm volatile("st.shared.f32 [%0], %1;" ::"r"(fo), "f"(acc.x * t0) : "memory");
+                    asm volatile("st.shared.f32 [%0], %1;" ::"r"(fo + FPITCH), "f"(acc.y * t1) : "memory");
+                    asm volatile("st.shared.f32 [%0], %1;" ::"r"(fo + 32), "f"(acc.z * t0) : "memory");
+                    asm volatile("st.shared.f32 [%0], %1;" ::"r"(fo + FPITCH + 32), "f"(acc.w * t1) : "memory");
+                    continue;
+                }
                 const uint32_t yo = ystage + m0 * YPITCH + (rb * 16 + r) * 2;
                 const __nv_bfloat16 o0 = __float2bfloat16_rn(acc.x * t0), o1 = __float2bfloat16_rn(acc.y * t1);
                 const __nv_bfloat16 o2 = __float2bfloat16_rn(acc.z * t0), o3 = __float2bfloat16_rn(acc.w * t1);
-                if (FUSE) {
+                if (SILU) {
                     // (o0, o2) = (gate, up) of channel 8 rb + r for token m0, (o1, o3) for token m0 + 1
                     const uint32_t h0 = silu_mul_bf16_bits(__bfloat162float(o0), __bfloat162float(o2));
                     const uint32_t h1 = silu_mul_bf16_bits(__bfloat162float(o1), __bfloat162float(o3));
@@ -606,7 +635,30 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
             }
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(part_empty);
-            if (has_start && !FUSE) {
+            if (has_start && with_res) {
+                constexpr int CPR = R / 8;
+#pragma unroll
+                for (int k = 0; k < RES_CHUNKS; ++k) {
+                    const int c = lane + 32 * k, m = c / CPR, col = c - m * CPR;
+                    if (c < a.M * CPR) {
+                        const float4 f0 = ptx::lds128f(ystage + m * FPITCH + col * 32), f1 = ptx::lds128f(ystage + m * FPITCH + col * 32 + 16);
+                        const uint4 rr = rv[k];
+                        uint4 v;
+                        __nv_bfloat162 b;
+                        b = __floats2bfloat162_rn(f0.x + __uint_as_float(rr.x << 16), f0.y + __uint_as_float(rr.x & 0xFFFF0000u));
+                        v.x = *reinterpret_cast<uint32_t*>(&b);
+                        b = __floats2bfloat162_rn(f0.z + __uint_as_float(rr.y << 16), f0.w + __uint_as_float(rr.y & 0xFFFF0000u));
+                        v.y = *reinterpret_cast<uint32_t*>(&b);
+                        b = __floats2bfloat162_rn(f1.x + __uint_as_float(rr.z << 16), f1.y + __uint_as_float(rr.z & 0xFFFF0000u));
+                        v.z = *reinterpret_cast<uint32_t*>(&b);
+                        b = __floats2bfloat162_rn(f1.z + __uint_as_float(rr.w << 16), f1.w + __uint_as_float(rr.w & 0xFFFF0000u));
+                        v.w = *reinterpret_cast<uint32_t*>(&b);
+                        *reinterpret_cast<uint4*>(a.y + (size_t)m * a.N + (size_t)strip * R + col * 8) = v;
+                    }
+                }
+                __syncwarp();
+            }
+            if (has_start && FUSE == 0) {
                 // the strip leaves in 16-byte pieces: R / 8 per token row
                 constexpr int CPR = R / 8;
                 for (int c = lane; c < a.M * CPR; c += 32) {
@@ -616,7 +668,7 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
                 }
                 __syncwarp();
             }
-            if (has_start && FUSE) {
+            if (has_start && SILU) {
                 // the strip's R / 2 channels of h, 16-byte pieces
                 constexpr int CPR = R / 16;
                 const int I = a.N / 2;
@@ -628,7 +680,7 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_const
                 __syncwarp();
             }
         }
-        if (FUSE) {
+        if (SILU) {
             // largest |h| per token over this CTA's strips: lanes of equal j hold the same two tokens
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb)
@@ -737,15 +789,16 @@ struct FuseOut {
 
 template <int MB, int RBLK, bool DEBUG, int FUSE>
 cudaError_t launch_strip(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed, void* y,
-                         int M, int N, int K, int ctas, void* workspace, int32_t* debug_partials, const FuseOut* fuse,
-                         cudaStream_t stream) {
+                         const void* residual, int M, int N, int K, int ctas, void* workspace, int32_t* debug_partials,
+                         const FuseOut* fuse, cudaStream_t stream) {
     constexpr int R = 16 * RBLK, GS = ST_UNITS / RBLK, MP = 8 * MB;
     const int G = K / GROUP;
-    const int fixed = st_layout(MB, RBLK, 0, G).total + 1024;
+    const bool fp32_stage = FUSE == 3;
+    const int fixed = st_layout(MB, RBLK, 0, G, fp32_stage).total + 1024;
     int stages = (ST_SMEM_BUDGET - fixed) / st_stage_bytes(MB, RBLK);
     if (stages > ST_MAX_STAGES) stages = ST_MAX_STAGES;
     if (stages < 2) return cudaErrorInvalidConfiguration;
-    const size_t smem = (size_t)st_layout(MB, RBLK, stages, G).total + 1024;
+    const size_t smem = (size_t)st_layout(MB, RBLK, stages, G, fp32_stage).total + 1024;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -789,6 +842,7 @@ cudaError_t launch_strip(const int8_t* qa, const uint16_t* sa, const int32_t* as
     a.status = reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF);
     a.slots = reinterpret_cast<unsigned long long*>(ws + WS_HEADER_BYTES);
     a.debug_partials = debug_partials;
+    a.residual = static_cast<const __nv_bfloat16*>(residual);
     a.h = fuse ? static_cast<__nv_bfloat16*>(fuse->h) : nullptr;
     a.qa_h = fuse ? fuse->qa_h : nullptr;
     a.sa_h = fuse ? fuse->sa_h : nullptr;
@@ -817,19 +871,23 @@ cudaError_t launch_strip(const int8_t* qa, const uint16_t* sa, const int32_t* as
 
 template <int MB, int RBLK>
 cudaError_t launch_strip_dbg(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed, void* y,
-                             int M, int N, int K, int ctas, void* workspace, int32_t* debug_partials, const FuseOut* fuse,
+                             const void* residual, int M, int N, int K, int ctas, void* workspace, int32_t* debug_partials, const FuseOut* fuse,
                              cudaStream_t stream) {
     if (fuse) {
         // two token blocks always run on 32-row strips (strip_plan): the other widths are not built in the fused form
         if constexpr (MB == 2 && RBLK != 2) return cudaErrorInvalidConfiguration;
         else if (fuse->one_kernel)
-            return launch_strip<MB, RBLK, false, 1>(qa, sa, asum, packed, nullptr, M, N, K, ctas, workspace, nullptr, fuse, stream);
+            return launch_strip<MB, RBLK, false, 1>(qa, sa, asum, packed, nullptr, nullptr, M, N, K, ctas, workspace, nullptr, fuse, stream);
         else
-            return launch_strip<MB, RBLK, false, 2>(qa, sa, asum, packed, nullptr, M, N, K, ctas, workspace, nullptr, fuse, stream);
+            return launch_strip<MB, RBLK, false, 2>(qa, sa, asum, packed, nullptr, nullptr, M, N, K, ctas, workspace, nullptr, fuse, stream);
+    }
+    if (residual) {                                      // its own instantiation: the plain kernel's epilogue stays as small as it was
+        if constexpr (MB == 2 && RBLK != 2) return cudaErrorInvalidConfiguration;
+        else return launch_strip<MB, RBLK, false, 3>(qa, sa, asum, packed, y, residual, M, N, K, ctas, workspace, nullptr, nullptr, stream);
     }
     if (debug_partials)
-        return launch_strip<MB, RBLK, true, 0>(qa, sa, asum, packed, y, M, N, K, ctas, workspace, debug_partials, nullptr, stream);
-    return launch_strip<MB, RBLK, false, 0>(qa, sa, asum, packed, y, M, N, K, ctas, workspace, nullptr, nullptr, stream);
+        return launch_strip<MB, RBLK, true, 0>(qa, sa, asum, packed, y, nullptr, M, N, K, ctas, workspace, debug_partials, nullptr, stream);
+    return launch_strip<MB, RBLK, false, 0>(qa, sa, asum, packed, y, nullptr, M, N, K, ctas, workspace, nullptr, nullptr, stream);
 }
 
 }  // namespace
@@ -885,12 +943,12 @@ void strip_plan(int M, int N, int K, int* strip_rows, int* ctas) {
 
 namespace {
 cudaError_t strip_dispatch(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
-                           void* y, int M, int N, int K, void* workspace, int32_t* debug_partials, const FuseOut* fuse,
+                           void* y, const void* residual, int M, int N, int K, void* workspace, int32_t* debug_partials, const FuseOut* fuse,
                            cudaStream_t stream) {
     int R = 0, ctas = 0;
     strip_plan(M, N, K, &R, &ctas);
 #define W4A8_STRIP_CASE(MBV, RBV) \
-    return launch_strip_dbg<MBV, RBV>(qa, sa, asum, packed, y, M, N, K, ctas, workspace, debug_partials, fuse, stream)
+    return launch_strip_dbg<MBV, RBV>(qa, sa, asum, packed, y, residual, M, N, K, ctas, workspace, debug_partials, fuse, stream)
     if (M <= 8) {
         if (R == 128) W4A8_STRIP_CASE(1, 8);
         if (R == 64) W4A8_STRIP_CASE(1, 4);
@@ -906,9 +964,9 @@ cudaError_t strip_dispatch(const int8_t* qa, const uint16_t* sa, const int32_t* 
 }  // namespace
 
 cudaError_t launch_gemm_strip(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
-                              void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
+                              void* y, const void* residual, int M, int N, int K, void* workspace, int32_t* debug_partials,
                               cudaStream_t stream) {
-    return strip_dispatch(qa, sa, asum, packed, y, M, N, K, workspace, debug_partials, nullptr, stream);
+    return strip_dispatch(qa, sa, asum, packed, y, residual, M, N, K, workspace, debug_partials, nullptr, stream);
 }
 
 // The fused gate+up form: packed = the 2 I = N channels in runs of eight gate / eight up; outputs h [M, I] bf16 and the
@@ -917,7 +975,7 @@ cudaError_t launch_gemm_strip_gate_up(const int8_t* qa, const uint16_t* sa, cons
                                       int M, int N, int K, void* h, int8_t* qa_h, uint16_t* sa_h, int32_t* asum_h,
                                       bool one_kernel, void* workspace, cudaStream_t stream) {
     const FuseOut f = {h, qa_h, sa_h, asum_h, one_kernel};
-    return strip_dispatch(qa, sa, asum, packed, nullptr, M, N, K, workspace, nullptr, &f, stream);
+    return strip_dispatch(qa, sa, asum, packed, nullptr, nullptr, M, N, K, workspace, nullptr, &f, stream);
 }
 
 }  // namespace w4a8

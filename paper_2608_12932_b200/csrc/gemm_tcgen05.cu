@@ -122,11 +122,13 @@ __device__ __forceinline__ uint32_t sub_zero4(uint32_t q, uint32_t kz) {
 // PC ("per channel"): the scales of a channel are the same in every group, so the integer sums of all
 // groups of a tile add up in one accumulator and the tile is drained once (see w4a8_gemm_per_channel).
 // BAL: balanced walk (see `segment` below).
-template <int TILE_M, bool DEBUG, bool SPLIT, bool PC = false, bool BAL = false>
+// RES: the epilogue adds a residual (its own instantiations: the extra registers of the residual block would
+// otherwise spill in the plain kernels).
+template <int TILE_M, bool DEBUG, bool SPLIT, bool PC = false, bool BAL = false, bool RES = false>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_constant__ CUtensorMap tmap_y,
                     const uint8_t* __restrict__ packed,
-                    const uint16_t* __restrict__ sa, __nv_bfloat16* __restrict__ y,
+                    const uint16_t* __restrict__ sa, __nv_bfloat16* y, const __nv_bfloat16* residual,
                     int32_t* __restrict__ debug_partials, uint32_t* __restrict__ status,
                     int M, int N, int K, int m_tiles, int total_tiles, int S,
                     float* __restrict__ handover, uint32_t* __restrict__ handover_flags) {
@@ -573,12 +575,31 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                     const float4 t = *reinterpret_cast<const float4*>(sa_w + b2 * 32 + 4 * k);
                     sc[4 * k] = t.x; sc[4 * k + 1] = t.y; sc[4 * k + 2] = t.z; sc[4 * k + 3] = t.w;
                 }
+                if (RES) {
+                    // the projection's output joins the residual stream: r[token][this lane's channel], added in fp32 before
+                    // the one rounding; folded into the scale registers' place (value = facc * sc + r) one token at a time.
+                    // y may be the residual buffer itself: this warp reads a block before it stores it.
+                    const __nv_bfloat16* rcol = residual + (size_t)ntile * TILE_N + q * 32 + lane;
+                    float rs[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int m = m_base + b2 * 32 + i;
+                        rs[i] = (b2 * 32 + i < C::W && m < M) ? __bfloat162float(rcol[(size_t)m * N]) : 0.0f;
+                    }
+                    if (lane == 0) ptx::bulk_wait_group_read0();
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (b2 * 32 + i < C::W)
+                            reinterpret_cast<__nv_bfloat16*>(ob + i * 64)[lane] = __float2bfloat16_rn(facc[b2 * 32 + i] * sc[i] + rs[i]);
+                } else {
                 if (lane == 0) ptx::bulk_wait_group_read0();      // the previous block's TMA store has read `ob`
                 __syncwarp();
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
                     if (b2 * 32 + i < C::W)
                         reinterpret_cast<__nv_bfloat16*>(ob + i * 64)[lane] = __float2bfloat16_rn(facc[b2 * 32 + i] * sc[i]);
+                }
                 if (b2 < C::NCH - 1 || C::LAST == 32) {
                     // a full block of 32 tokens: one TMA store (rows past M are clipped by the map), the warp moves on
                     ptx::fence_proxy_async_smem();
@@ -621,7 +642,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                 const int idx = lo + i, m = mtile * TILE_M + idx / TILE_N, nn = idx % TILE_N;
                 if (m < M) {
                     const float t = __half2float(__ushort_as_half(__ldg(sa + m)));
-                    y[(size_t)m * N + (size_t)ntile * TILE_N + nn] = __float2bfloat16_rn(acc * t);
+                    float v = acc * t;
+                    if (RES) v += __bfloat162float(residual[(size_t)m * N + (size_t)ntile * TILE_N + nn]);
+                    y[(size_t)m * N + (size_t)ntile * TILE_N + nn] = __float2bfloat16_rn(v);
                 }
             }
         }
@@ -635,8 +658,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
     }
 }
 
-template <int TILE_M, bool DEBUG, bool SPLIT, bool PC = false, bool BAL = false>
-cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed, void* y, int M, int N, int K, int S,
+template <int TILE_M, bool DEBUG, bool SPLIT, bool PC = false, bool BAL = false, bool RES = false>
+cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed, void* y, const void* residual, int M, int N, int K, int S,
                         void* workspace, int32_t* debug_partials, cudaStream_t stream) {
     using C = Cfg<TILE_M>;
     CUtensorMap tmap, tmap_y;
@@ -652,7 +675,7 @@ cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     const int sms = device_sm_count();
     if (!attr_done[dev]) {
-        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT, PC, BAL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT, PC, BAL, RES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  C::SMEM_ALLOC);
         if (e != cudaSuccess) return e;
         attr_done[dev] = true;
@@ -677,8 +700,9 @@ cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT, PC, BAL>, tmap, tmap_y, static_cast<const uint8_t*>(packed), sa,
-                              static_cast<__nv_bfloat16*>(y), debug_partials, reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF),
+    return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT, PC, BAL, RES>, tmap, tmap_y, static_cast<const uint8_t*>(packed), sa,
+                              static_cast<__nv_bfloat16*>(y), static_cast<const __nv_bfloat16*>(residual), debug_partials,
+                              reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF),
                               M, N, K, m_tiles, total, S, reinterpret_cast<float*>(ws + WS_SHARED_OFF),
                               reinterpret_cast<uint32_t*>(ws + WS_COUNTER_OFF));
 }
@@ -713,22 +737,22 @@ int max_active_clusters(int S) {
     return cached[dev][S] > 0 ? cached[dev][S] : 0;
 }
 
-template <bool DEBUG, bool PC = false>
+template <bool DEBUG, bool PC = false, bool RES = false>
 cudaError_t launch_plan(int tile_m, int S, bool balanced, const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
-                        int M, int N, int K, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
+                        const void* residual, int M, int N, int K, void* workspace, int32_t* debug_partials, cudaStream_t stream) {
     if (S > 1 && !PC) {
-        if (tile_m == 64) return launch_tile<64, DEBUG, true>(qa, sa, packed, y, M, N, K, S, workspace, debug_partials, stream);
-        if (tile_m == 128) return launch_tile<128, DEBUG, true>(qa, sa, packed, y, M, N, K, S, workspace, debug_partials, stream);
-        return launch_tile<208, DEBUG, true>(qa, sa, packed, y, M, N, K, S, workspace, debug_partials, stream);
+        if (tile_m == 64) return launch_tile<64, DEBUG, true, false, false, RES>(qa, sa, packed, y, residual, M, N, K, S, workspace, debug_partials, stream);
+        if (tile_m == 128) return launch_tile<128, DEBUG, true, false, false, RES>(qa, sa, packed, y, residual, M, N, K, S, workspace, debug_partials, stream);
+        return launch_tile<208, DEBUG, true, false, false, RES>(qa, sa, packed, y, residual, M, N, K, S, workspace, debug_partials, stream);
     }
     if (balanced && !PC) {
-        if (tile_m == 64) return launch_tile<64, DEBUG, false, false, true>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
-        if (tile_m == 128) return launch_tile<128, DEBUG, false, false, true>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
-        return launch_tile<208, DEBUG, false, false, true>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
+        if (tile_m == 64) return launch_tile<64, DEBUG, false, false, true, RES>(qa, sa, packed, y, residual, M, N, K, 1, workspace, debug_partials, stream);
+        if (tile_m == 128) return launch_tile<128, DEBUG, false, false, true, RES>(qa, sa, packed, y, residual, M, N, K, 1, workspace, debug_partials, stream);
+        return launch_tile<208, DEBUG, false, false, true, RES>(qa, sa, packed, y, residual, M, N, K, 1, workspace, debug_partials, stream);
     }
-    if (tile_m == 64) return launch_tile<64, DEBUG, false, PC>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
-    if (tile_m == 128) return launch_tile<128, DEBUG, false, PC>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
-    return launch_tile<208, DEBUG, false, PC>(qa, sa, packed, y, M, N, K, 1, workspace, debug_partials, stream);
+    if (tile_m == 64) return launch_tile<64, DEBUG, false, PC, false, RES>(qa, sa, packed, y, residual, M, N, K, 1, workspace, debug_partials, stream);
+    if (tile_m == 128) return launch_tile<128, DEBUG, false, PC, false, RES>(qa, sa, packed, y, residual, M, N, K, 1, workspace, debug_partials, stream);
+    return launch_tile<208, DEBUG, false, PC, false, RES>(qa, sa, packed, y, residual, M, N, K, 1, workspace, debug_partials, stream);
 }
 
 }  // namespace
@@ -772,14 +796,16 @@ long tcgen05_plan(int M, int N, int K, int sms, int* tile_m, int* split, int max
     return best_ns;                                                   // the estimate, for the caller's choice of kernel family
 }
 
-cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
+cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void* packed, void* y, const void* residual,
                                 int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream) {
     int tile_m = 64, S = 1, balanced = 0;
     tcgen05_plan(M, N, K, device_sm_count(), &tile_m, &S, TC_MAX_SPLIT, &balanced);
+    if (residual)                                   // (no partials dump in this form)
+        return launch_plan<false, false, true>(tile_m, S, balanced != 0, qa, sa, packed, y, residual, M, N, K, workspace, nullptr, stream);
     if (debug_partials)
-        return launch_plan<true>(tile_m, S, balanced != 0, qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
-    return launch_plan<false>(tile_m, S, balanced != 0, qa, sa, packed, y, M, N, K, workspace, debug_partials, stream);
+        return launch_plan<true>(tile_m, S, balanced != 0, qa, sa, packed, y, nullptr, M, N, K, workspace, debug_partials, stream);
+    return launch_plan<false>(tile_m, S, balanced != 0, qa, sa, packed, y, nullptr, M, N, K, workspace, debug_partials, stream);
 }
 
 // The same pipeline with one drain per tile: for weights whose scale does not change along K.
@@ -790,8 +816,8 @@ cudaError_t launch_gemm_tcgen05_per_channel(const int8_t* qa, const uint16_t* sa
     int tile_m = 64, S = 1;
     tcgen05_plan(M, N, K, device_sm_count(), &tile_m, &S, 1, nullptr);
     if (debug_sums)
-        return launch_plan<true, true>(tile_m, 1, false, qa, sa, packed, y, M, N, K, workspace, debug_sums, stream);
-    return launch_plan<false, true>(tile_m, 1, false, qa, sa, packed, y, M, N, K, workspace, debug_sums, stream);
+        return launch_plan<true, true>(tile_m, 1, false, qa, sa, packed, y, nullptr, M, N, K, workspace, debug_sums, stream);
+    return launch_plan<false, true>(tile_m, 1, false, qa, sa, packed, y, nullptr, M, N, K, workspace, debug_sums, stream);
 }
 
 }  // namespace w4a8

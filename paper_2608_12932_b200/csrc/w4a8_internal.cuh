@@ -93,7 +93,7 @@ static_assert(WS_HEADER_BYTES + STRIP_MAX_CTAS * STRIP_SLOT_BYTES == W4A8_WORKSP
 bool strip_supported(int M, int N, int K);
 void strip_plan(int M, int N, int K, int* strip_rows, int* ctas);
 cudaError_t launch_gemm_strip(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
-                              void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
+                              void* y, const void* residual, int M, int N, int K, void* workspace, int32_t* debug_partials,
                               cudaStream_t stream);
 // W4A16 (bf16 activations against the same packed weights), up to STRIP_MAX_M tokens
 bool a16_supported(int M, int N, int K);
@@ -109,10 +109,11 @@ cudaError_t launch_gemm_strip_gate_up(const int8_t* qa, const uint16_t* sa, cons
                                       bool one_kernel, void* workspace, cudaStream_t stream);
 int device_sm_count();                       // SMs of the current device (cached per device)
 int cluster_num_slices(int M, int N, int K);
+// residual: null, or bf16 [M,N] added to the projection before the one rounding (may be y itself)
 cudaError_t launch_gemm_cluster(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
-                                void* y, int M, int N, int K, void* workspace, int32_t* debug_partials,
+                                void* y, const void* residual, int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream);
-cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
+cudaError_t launch_gemm_tcgen05(const int8_t* qa, const uint16_t* sa, const void* packed, void* y, const void* residual,
                                 int M, int N, int K, void* workspace, int32_t* debug_partials,
                                 cudaStream_t stream);
 cudaError_t launch_gemm_tcgen05_per_channel(const int8_t* qa, const uint16_t* sa, const void* packed, void* y,
