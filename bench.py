@@ -485,9 +485,10 @@ def run_layer_chain(torch, B, peaks, l2_bytes, timer):
                          step_bytes(M, L["N"], L["K"]) / (peaks["hbm_gbs"] * 1e9)) for L in layers)
         row = {"M": M, "us_per_layer": round(us, 2), "kernels_per_layer": 8, "tops": round(ops / us / 1e6, 1),
                "gbs": round(nbytes / us / 1e3, 1), "frac_measured": round(t_roof * 1e6 / us, 3)}
-        # The same layer with the fused gate+up step: the projection's epilogue (or, above 16 tokens, the quantiser that
+        # The same layer with the fused steps: the gate+up projection's epilogue (or, above 16 tokens, the quantiser that
         # follows it) forms SiLU(gate) * up and the down projection's quantised input, which the down projection then
-        # takes as it is - the real data dependency of a decoder layer, one kernel fewer where the fusion is one kernel.
+        # takes as it is - the real data dependency of a decoder layer; O and down add their output into the residual
+        # stream in their epilogues, in place.
         # Fractions use the same roofline sum as above (the same logical work).
         by_name = dict(zip(wl.LAYERS.keys(), layers))
         gu, dn = by_name["gate_up"], by_name["down"]
@@ -495,6 +496,8 @@ def run_layer_chain(torch, B, peaks, l2_bytes, timer):
         assert dn["K"] == I
         h_out = (torch.empty((M, I), dtype=torch.bfloat16, device="cuda"), torch.empty((M, I), dtype=torch.int8, device="cuda"),
                  torch.empty((M,), dtype=torch.float16, device="cuda"), torch.empty((M, I // 128), dtype=torch.int32, device="cuda"))
+        resid = torch.zeros((M, dn["N"]), dtype=torch.bfloat16, device="cuda")
+        assert by_name["o"]["N"] == dn["N"]
         form_names = {B.GATE_UP_EPILOGUE: "SiLU*up in the strip kernel's epilogue + requantise kernel",
                       B.GATE_UP_ONE_KERNEL: "one kernel (epilogue, last CTAs stay and requantise)",
                       B.GATE_UP_SEPARATE: "GEMM + SiLU*up quantiser"}
@@ -503,13 +506,16 @@ def run_layer_chain(torch, B, peaks, l2_bytes, timer):
             def body_fused():
                 for _ in range(reps):
                     for c in range(ncopies):
-                        for name in ("qkv", "o"):
-                            L = by_name[name]
-                            B.w4a8_linear(L["xm"], L["packed"][c], L["N"], L["ws"], 128, out=L["y"], scratch=L["scratch"])
+                        L = by_name["qkv"]
+                        B.w4a8_linear(L["xm"], L["packed"][c], L["N"], L["ws"], 128, out=L["y"], scratch=L["scratch"])
+                        L = by_name["o"]                       # O and down add into the residual stream, in place
+                        B.w4a8_quantize_act(L["xm"], 128, out=L["scratch"])
+                        B.w4a8_gemm_residual(L["scratch"][0], L["scratch"][1], L["scratch"][2], L["packed"][c], resid, L["N"], L["ws"],
+                                             128, out=resid)
                         B.w4a8_quantize_act(gu["xm"], 128, out=gu["scratch"])
                         B.w4a8_gate_up_silu_quantize(gu["scratch"][0], gu["scratch"][1], gu["scratch"][2], gu["packed"][c], gu["N"],
                                                      gu["ws"], 128, form=form, y_scratch=gu["y"], out=h_out)
-                        B.w4a8_gemm(h_out[1], h_out[2], h_out[3], dn["packed"][c], dn["N"], dn["ws"], 128, out=dn["y"])
+                        B.w4a8_gemm_residual(h_out[1], h_out[2], h_out[3], dn["packed"][c], resid, dn["N"], dn["ws"], 128, out=resid)
             _, times = timer.graph_ms(body_fused, replays=5, warm=2)
             for L in layers:
                 B.w4a8_check_status(L["ws"])

@@ -434,6 +434,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
             float facc[C::W];
 #pragma unroll
             for (int i = 0; i < C::W; ++i) facc[i] = 0.0f;
+            if (RES) {
+                // the residual of this warp's part of the tile (W tokens x 64 bytes) is asked into L2 now; the epilogue's
+                // loads then find it there
+#pragma unroll
+                for (int k = 0; k < C::NCH; ++k) {
+                    const int m = m_base + lane + 32 * k;
+                    if (lane + 32 * k < C::W && m < M)
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(residual + (size_t)m * N + (size_t)ntile * TILE_N + q * 32));
+                }
+            }
             // this warp's token scales, widened once per tile (rows past M get 0 and are never stored)
             float* sa_w = reinterpret_cast<float*>(smem + C::SA_OFF) + (warp - WARP_DRAIN0) * (C::NCH * 32);
             __syncwarp();
@@ -564,6 +574,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
             uint8_t* ob = smem + C::OUT_OFF + (warp - WARP_DRAIN0) * 2048;
             const uint32_t ob_addr = smem_base + C::OUT_OFF + (warp - WARP_DRAIN0) * 2048;
             __nv_bfloat16* yrow = y + (size_t)ntile * TILE_N + q * 32 + 8 * (lane & 3);
+            uint4 rv[4];
+            // residual rows 8 k + lane / 4 of block b, this lane's 16-byte piece of the warp's 64-byte row (zeros past M or W)
+            auto load_res = [&](int b, uint4 (&dst)[4]) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int t = b * 32 + 8 * k + (lane >> 2), m = m_base + t;
+                    dst[k] = make_uint4(0u, 0u, 0u, 0u);
+                    if (RES && t < C::W && m < M)
+                        dst[k] = __ldcg(reinterpret_cast<const uint4*>(residual + (size_t)m * N + (size_t)ntile * TILE_N + q * 32 + 8 * (lane & 3)));
+                }
+            };
 #pragma unroll
             for (int b2 = 0; b2 < C::NCH; ++b2) {
                 // The chunk's 32 token scales go to registers first: read one by one between the stores below
@@ -576,22 +597,34 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                     sc[4 * k] = t.x; sc[4 * k + 1] = t.y; sc[4 * k + 2] = t.z; sc[4 * k + 3] = t.w;
                 }
                 if (RES) {
-                    // the projection's output joins the residual stream: r[token][this lane's channel], added in fp32 before
-                    // the one rounding; folded into the scale registers' place (value = facc * sc + r) one token at a time.
-                    // y may be the residual buffer itself: this warp reads a block before it stores it.
-                    const __nv_bfloat16* rcol = residual + (size_t)ntile * TILE_N + q * 32 + lane;
-                    float rs[32];
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int m = m_base + b2 * 32 + i;
-                        rs[i] = (b2 * 32 + i < C::W && m < M) ? __bfloat162float(rcol[(size_t)m * N]) : 0.0f;
-                    }
+                    // The projection's output joins the residual stream, added in fp32 before the one rounding.  A block's
+                    // residual (32 tokens x this warp's 32 channels) is fetched in the layout of the stores - 16 bytes per
+                    // lane, rows of 64 bytes, one block ahead - and written into the output block, from which each lane
+                    // reads its own channel's column back, adds, rounds and overwrites.  y may be the residual buffer:
+                    // this warp reads a block before it stores it.
+                    if (b2 == 0) load_res(0, rv);
+                    uint4 rv_next[4];
+                    if (b2 + 1 < C::NCH) load_res(b2 + 1, rv_next);
                     if (lane == 0) ptx::bulk_wait_group_read0();
                     __syncwarp();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (b2 * 32 + i < C::W)
-                            reinterpret_cast<__nv_bfloat16*>(ob + i * 64)[lane] = __float2bfloat16_rn(facc[b2 * 32 + i] * sc[i] + rs[i]);
+                    for (int k = 0; k < 4; ++k)
+                        *reinterpret_cast<uint4*>(ob + (8 * k + (lane >> 2)) * 64 + 16 * (lane & 3)) = rv[k];
+                    __syncwarp();
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        float rs[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            rs[i] = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(ob + (16 * half + i) * 64)[lane]);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            if (b2 * 32 + 16 * half + i < C::W)
+                                reinterpret_cast<__nv_bfloat16*>(ob + (16 * half + i) * 64)[lane] =
+                                    __float2bfloat16_rn(facc[b2 * 32 + 16 * half + i] * sc[16 * half + i] + rs[i]);
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) rv[k] = rv_next[k];
                 } else {
                 if (lane == 0) ptx::bulk_wait_group_read0();      // the previous block's TMA store has read `ob`
                 __syncwarp();
