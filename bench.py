@@ -442,6 +442,32 @@ def run_w4a16_comparison(torch, B, peaks, l2_bytes, timer):
     return rows
 
 
+def run_rope_roofline(torch, B, peaks, l2_bytes, timer):
+    """Rotary embedding of pre-rotation cached keys at shifted positions (streaming prefill): 8 KV heads of 128, a window
+    of 4096 tokens and a long one of 65536; inputs visited in turn (more than two L2 capacities in all)."""
+    rows = []
+    for T in (4096, 65536):
+        H, D = 8, 128
+        nbytes = T * H * D * 4 + 4 * T
+        ncopies = copies_for(T * H * D * 2, l2_bytes)
+        ks = [torch.randn((T, H, D), device="cuda").to(torch.bfloat16) for _ in range(ncopies)]
+        pos = torch.arange(T, dtype=torch.int32, device="cuda")
+        out = torch.empty_like(ks[0])
+
+        def body():
+            for k in ks:
+                B.w4a8_rope_shifted_keys(k, pos, 45, 1.0e6, out=out)
+        _, times = timer.graph_ms(body, replays=5, warm=2)
+        us = float(np.median(times)) * 1e3 / ncopies
+        rows.append({"kernel": "rope_shifted_keys_kernel", "workload": f"T={T} H={H} D={D}", "bound": "hbm",
+                     "achieved": round(nbytes / us / 1e3, 1), "unit": "GB/s", "peak": peaks["hbm_gbs"],
+                     "frac": round(nbytes / us / 1e3 / peaks["hbm_gbs"], 4), "us_per_launch": round(us, 2),
+                     "algorithmic_bytes_per_launch": nbytes})
+        del ks
+        torch.cuda.empty_cache()
+    return rows
+
+
 def run_layer_chain(torch, B, peaks, l2_bytes, timer):
     """The four linears of one decoder layer back to back (QKV, O, gate+up, down), each as the public
     w4a8_linear call (quantise + GEMM) on its own input, in one CUDA graph: what a decoder layer spends in
@@ -675,6 +701,7 @@ def run_gpu(args):
     peaks.update(measure_int8_peak(torch))
     roof_large = run_large_m_roofline(torch, B, peaks, l2_bytes, timer)
     roof_quant = run_quantize_roofline(torch, B, peaks, l2_bytes, timer)
+    roof_rope = run_rope_roofline(torch, B, peaks, l2_bytes, timer)
 
     sweep = None
     targets = None
@@ -719,6 +746,7 @@ def run_gpu(args):
         "peaks": {k: (round(v, 1) if isinstance(v, float) else v) for k, v in peaks.items()},
         "roofline_large_m": roof_large,
         "roofline_quantize_act": roof_quant,
+        "roofline_rope_shifted_keys": roof_rope,
     }
     if sweep is not None:
         line["targets"] = targets

@@ -230,6 +230,29 @@ w4a8_status w4a8_gate_up_silu_quantize(int form, const int8_t* qa, const uint16_
                                        void* stream);
 
 /*
+ * Two pieces of streaming prefill that sit beside the quantised linears (Sec. 3.1, "Streaming design").
+ *
+ * w4a8_rope_shifted_keys: keys are cached before the rotary embedding, because a cached token's position changes
+ * when the window slides; the rotation is applied at use, at the shifted position pos[t] - delta.  Rotate-half
+ * form (this library's reading; the paper names no variant): for i < D/2, theta_i = base^(-2i/D),
+ * phi = (pos[t] - delta) theta_i,
+ *   out[t,h,i] = k[t,h,i] cos(phi) - k[t,h,i+D/2] sin(phi),  out[t,h,i+D/2] = k[t,h,i+D/2] cos(phi) + k[t,h,i] sin(phi)
+ * The angle is formed and reduced in fp64, sine, cosine, products and sums are fp32, one rounding to bf16 (equal to
+ * the fp64 definition's bf16 or its neighbour).
+ *   k_pre, k_rot  device, bf16 [T,H,D] row-major, 4-byte aligned (may be the same buffer: a thread reads the four
+ *                 values it then writes);  pos  device, int32 [T];  D % 4 == 0;  base > 1 (e.g. 1e6)
+ *
+ * w4a8_streaming_mask: the new frame's tokens take the last-frame place of each camera view (the sequence is
+ * view-major: all frames of one view before the next), only they are queries, attention stays causal in that order:
+ *   mask[q][j] = 1 iff j <= position of query q,  query q = (view v, token i) at position (v frames + frames - 1) n + i
+ *   mask  device, uint8 [views * n, views * frames * n] row-major.  (The paper's figure of the mask is not
+ *   available; this is its caption written out.)
+ */
+w4a8_status w4a8_rope_shifted_keys(const void* k_pre_bf16, const int32_t* pos, int delta, int T, int H, int D,
+                                   double base, void* k_rot_bf16, void* stream);
+w4a8_status w4a8_streaming_mask(int views, int frames, int tokens_per_frame, uint8_t* mask, void* stream);
+
+/*
  * The weight-only variant the paper contrasts W4A8 with (Sec. 3.4, first paragraph: 4-bit weights with 16-bit
  * activations shrink what the memory-bound decode must load, and leave the arithmetic of the compute-bound
  * prefill in 16-bit floating point).  Same packed weights, activations NOT quantised:

@@ -23,7 +23,8 @@ EXPORTS = ("w4a8_status_string", "w4a8_packed_bytes", "w4a8_workspace_bytes", "w
            "w4a8_linear", "w4a8_linear_host", "w4a8_gemm_static_scratch", "w4a8_check_status", "w4a8_plan",
            "w4a8_gemm_per_channel", "w4a8_static_scratch_status", "w4a8_selftest_wait_timeout",
            "w4a8_silu_mul_quantize", "w4a8_gate_up_form", "w4a8_gate_up_silu_quantize", "w4a8_a16_gemm",
-           "w4a8_dequantize_weights", "w4a8_gemm_residual")
+           "w4a8_dequantize_weights", "w4a8_gemm_residual", "w4a8_rope_shifted_keys",
+           "w4a8_streaming_mask")
 
 _lib = None
 
@@ -67,6 +68,10 @@ def lib():
         L.w4a8_plan.argtypes = [ci, ci, ci, ci, vp]
         L.w4a8_silu_mul_quantize.restype = ci
         L.w4a8_silu_mul_quantize.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp]
+        L.w4a8_rope_shifted_keys.restype = ci
+        L.w4a8_rope_shifted_keys.argtypes = [vp, vp, ci, ci, ci, ci, ctypes.c_double, vp, vp]
+        L.w4a8_streaming_mask.restype = ci
+        L.w4a8_streaming_mask.argtypes = [ci, ci, ci, vp, vp]
         L.w4a8_gemm_residual.restype = ci
         L.w4a8_gemm_residual.argtypes = [ci, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp]
         L.w4a8_a16_gemm.restype = ci
@@ -282,6 +287,24 @@ def w4a8_gemm_residual(qa, sa, asum, packed_w, residual, N, workspace, group=GRO
     _check(lib().w4a8_gemm_residual(path, _ptr(qa), _ptr(sa), _ptr(asum), _ptr(packed_w), _ptr(residual), _ptr(out), M, N, K, group,
                                     _ptr(workspace), workspace.numel(), _stream(stream)), "w4a8_gemm_residual")
     return out
+
+
+def w4a8_rope_shifted_keys(k_pre, pos, delta, base, out=None, stream=None):
+    """k_pre bf16 [T,H,D], pos int32 [T] -> keys rotated at positions pos - delta (rotate-half rotary embedding)."""
+    _dev(k_pre, torch.bfloat16, "k_pre"), _dev(pos, torch.int32, "pos")
+    T, H, D = k_pre.shape
+    if out is None:
+        out = torch.empty_like(k_pre)
+    _check(lib().w4a8_rope_shifted_keys(_ptr(k_pre), _ptr(pos), int(delta), T, H, D, float(base), _ptr(out), _stream(stream)),
+           "w4a8_rope_shifted_keys")
+    return out
+
+
+def w4a8_streaming_mask(views, frames, tokens_per_frame, device="cuda", stream=None):
+    """uint8 [views * n, views * frames * n]: which keys the newest frame's tokens may attend."""
+    mask = torch.empty((views * tokens_per_frame, views * frames * tokens_per_frame), dtype=torch.uint8, device=device)
+    _check(lib().w4a8_streaming_mask(views, frames, tokens_per_frame, _ptr(mask), _stream(stream)), "w4a8_streaming_mask")
+    return mask
 
 
 def w4a8_a16_gemm(x, packed_w, N, workspace, group=GROUP, out=None, stream=None):

@@ -254,6 +254,27 @@ w4a8_status w4a8_gate_up_silu_quantize(int form, const int8_t* qa, const uint16_
     return launch_silu_mul_quantize(y_scratch_bf16, M, N / 2, h_bf16, qa_h, sa_h, asum_h, st) == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
 
+w4a8_status w4a8_rope_shifted_keys(const void* k_pre_bf16, const int32_t* pos, int delta, int T, int H, int D, double base,
+                                   void* k_rot_bf16, void* stream) {
+    if (T < 0 || H <= 0 || D <= 0 || D % 4 != 0 || !(base > 1.0)) return W4A8_ERR_SHAPE;
+    if (T == 0) return W4A8_OK;
+    if (!k_pre_bf16 || !pos || !k_rot_bf16) return W4A8_ERR_NULL;
+    if (!aligned(k_pre_bf16, 4) || !aligned(k_rot_bf16, 4) || !aligned(pos, 4)) return W4A8_ERR_ALIGN;
+    w4a8_status a = arch_check();
+    if (a != W4A8_OK) return a;
+    return launch_rope_shifted_keys(k_pre_bf16, pos, delta, T, H, D, base, k_rot_bf16, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+w4a8_status w4a8_streaming_mask(int views, int frames, int tokens_per_frame, uint8_t* mask, void* stream) {
+    if (views <= 0 || frames <= 0 || tokens_per_frame <= 0) return W4A8_ERR_SHAPE;
+    if (!mask) return W4A8_ERR_NULL;
+    w4a8_status a = arch_check();
+    if (a != W4A8_OK) return a;
+    return launch_streaming_mask(views, frames, tokens_per_frame, mask, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
 w4a8_status w4a8_a16_gemm(const void* x_bf16, const void* packed_w, void* y_bf16, int M, int N, int K, int group,
                           void* workspace, size_t workspace_bytes, void* stream) {
     if (!shape_ok(N, K, group) || M < 0) return W4A8_ERR_SHAPE;

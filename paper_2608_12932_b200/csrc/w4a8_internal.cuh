@@ -95,6 +95,10 @@ void strip_plan(int M, int N, int K, int* strip_rows, int* ctas);
 cudaError_t launch_gemm_strip(const int8_t* qa, const uint16_t* sa, const int32_t* asum, const void* packed,
                               void* y, const void* residual, int M, int N, int K, void* workspace, int32_t* debug_partials,
                               cudaStream_t stream);
+// streaming prefill: rotary embedding of pre-rotation cached keys at shifted positions; the streaming attention mask
+cudaError_t launch_rope_shifted_keys(const void* k_pre, const int32_t* pos, int delta, int T, int H, int D, double base,
+                                     void* k_rot, cudaStream_t stream);
+cudaError_t launch_streaming_mask(int V, int F, int n, uint8_t* mask, cudaStream_t stream);
 // W4A16 (bf16 activations against the same packed weights), up to STRIP_MAX_M tokens
 bool a16_supported(int M, int N, int K);
 void a16_plan(int M, int N, int K, int* strip_rows, int* ctas);
