@@ -226,7 +226,7 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-// 2-D tiled TMA load (no multicast); x = innermost coordinate (x * element size must be a multiple of 16 B)
+// 2-D tiled TMA load into this CTA alone; x = innermost coordinate (x * element size must be a multiple of 16 B)
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, int x, int y, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                  ::"r"(dst), "l"(tmap), "r"(bar), "r"(x), "r"(y) : "memory");
@@ -241,7 +241,7 @@ __device__ __forceinline__ void tma_prefetch_3d(const void* tmap, int x, int y, 
 __device__ __forceinline__ void tma_prefetch_4d(const void* tmap, int x, int y, int z, int w) {
     asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(tmap), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
 }
-// 3-D and 4-D tiled TMA loads (no multicast); same alignment rule for the innermost coordinate
+// 3-D and 4-D tiled TMA loads into this CTA alone; same alignment rule for the innermost coordinate
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, int x, int y, int z, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
                  ::"r"(dst), "l"(tmap), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
