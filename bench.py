@@ -777,13 +777,21 @@ def run_shape(args):
     packed = [packed0] + [packed0.clone() for _ in range(ncopies - 1)]
     ws = B.new_workspace(M, N, K)
     x = to_dev16(torch, case["x"], torch.bfloat16)
-    y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    h_out = (torch.empty((M, N // 2), dtype=torch.bfloat16, device="cuda"), torch.empty((M, N // 2), dtype=torch.int8, device="cuda"),
+             torch.empty((M,), dtype=torch.float16, device="cuda"), torch.empty((M, N // 256), dtype=torch.int32, device="cuda"))
     times = []
     for i in range(args.warmup + args.steps):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         qa, sa, asum = B.w4a8_quantize_act(x)
         e0.record()
-        if args.per_channel:
+        if args.variant == "a16":
+            B.w4a8_a16_gemm(x, packed[i % ncopies], N, ws, out=y)
+        elif args.variant == "gate_up":
+            B.w4a8_gate_up_silu_quantize(qa, sa, asum, packed[i % ncopies], N, ws, y_scratch=y, out=h_out)
+        elif args.variant == "residual":
+            B.w4a8_gemm_residual(qa, sa, asum, packed[i % ncopies], y, N, ws, out=y)
+        elif args.per_channel:
             B.w4a8_gemm_per_channel(qa, sa, packed[i % ncopies], N, ws, out=y)
         else:
             B.w4a8_gemm(qa, sa, asum, packed[i % ncopies], N, ws, out=y)
@@ -793,9 +801,36 @@ def run_shape(args):
             times.append(e0.elapsed_time(e1) * 1e3)
     B.w4a8_check_status(ws)
     us = float(np.median(times))
-    print(json.dumps({"shape": args.shape, "per_channel_scales": bool(args.per_channel), "M": M, "N": N, "K": K, "gemm_us_eager_median": round(us, 2),
+    print(json.dumps({"shape": args.shape, "variant": args.variant, "per_channel_scales": bool(args.per_channel), "M": M, "N": N, "K": K, "gemm_us_eager_median": round(us, 2),
                       "tops": round(wl.algorithmic_ops(M, N, K) / us / 1e6, 1),
                       "gbs": round(wl.algorithmic_bytes_gemm(M, N, K) / us / 1e3, 1), "launches": args.steps}))
+
+
+def run_rope(args):
+    """--rope T : w4a8_rope_shifted_keys on T tokens x 8 heads x 128, launched eagerly `steps` times on inputs visited
+    in turn (the small case that ncu captures are taken on); prints one JSON line."""
+    import torch
+
+    from paper_2608_12932_b200 import binding as B
+    T, H, D = args.rope, 8, 128
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    l2_bytes = torch.cuda.get_device_properties(torch.cuda.current_device()).L2_cache_size or L2_BYTES_ASSUMED
+    ncopies = copies_for(T * H * D * 2, l2_bytes)
+    ks = [torch.randn((T, H, D), device="cuda").to(torch.bfloat16) for _ in range(ncopies)]
+    pos = torch.arange(T, dtype=torch.int32, device="cuda")
+    out = torch.empty_like(ks[0])
+    times = []
+    for i in range(args.warmup + args.steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.w4a8_rope_shifted_keys(ks[i % ncopies], pos, 45, 1.0e6, out=out)
+        e1.record()
+        e1.synchronize()
+        if i >= args.warmup:
+            times.append(e0.elapsed_time(e1) * 1e3)
+    us = float(np.median(times))
+    print(json.dumps({"rope": {"T": T, "H": H, "D": D}, "us_eager_median": round(us, 2), "gbs": round(T * H * D * 4 / us / 1e3, 1),
+                      "launches": args.steps}))
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one GEMM launch at the headline shape, by kernel, from the ncu
@@ -814,9 +849,14 @@ def main():
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--shape", default=None, help="LAYER:M, e.g. gate_up:1024 - run only that GEMM (profiling aid)")
     ap.add_argument("--per-channel", action="store_true", help="with --shape: w4a8_gemm_per_channel instead of w4a8_gemm")
+    ap.add_argument("--variant", default="gemm", choices=["gemm", "a16", "gate_up", "residual"],
+                    help="with --shape: w4a8_a16_gemm, w4a8_gate_up_silu_quantize (gate_up layer) or w4a8_gemm_residual instead of w4a8_gemm")
+    ap.add_argument("--rope", type=int, default=0, help="T: run only w4a8_rope_shifted_keys on T tokens x 8 heads x 128 (profiling aid)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
-    if args.shape:
+    if args.rope:
+        run_rope(args)
+    elif args.shape:
         run_shape(args)
     elif args.impl == "reference":
         run_reference(args)
