@@ -64,7 +64,11 @@ namespace {
 constexpr int ST_CONSUMER_WARPS = ST_CW;
 constexpr int ST_UNITS = 2 * ST_CONSUMER_WARPS;           // units (16 rows x one group) per stage
 constexpr int ST_NIB_BYTES = ST_UNITS * 1024;             // nibbles of a stage
-constexpr int ST_PRODUCER_WARPS = 3;
+// three producer warps: two or four (-DST_PW) move every layer by less than 2 % either way
+#ifndef ST_PW
+#define ST_PW 3
+#endif
+constexpr int ST_PRODUCER_WARPS = ST_PW;
 constexpr int ST_EPILOGUE_WARP = ST_CONSUMER_WARPS + ST_PRODUCER_WARPS;
 constexpr int ST_THREADS = (ST_CONSUMER_WARPS + ST_PRODUCER_WARPS + 1) * 32;
 constexpr int ST_MAX_STAGES = 8;
