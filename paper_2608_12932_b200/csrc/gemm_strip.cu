@@ -72,8 +72,14 @@ constexpr int ST_PRODUCER_WARPS = ST_PW;
 constexpr int ST_EPILOGUE_WARP = ST_CONSUMER_WARPS + ST_PRODUCER_WARPS;
 constexpr int ST_THREADS = (ST_CONSUMER_WARPS + ST_PRODUCER_WARPS + 1) * 32;
 constexpr int ST_MAX_STAGES = 8;
-constexpr int ST_W_BYTES = ST_CW == 8 ? 17408 : 26624;                         // weight part of a stage (16 KB of nibbles + scales + zero points, padded)
-constexpr int ST_SMEM_BUDGET = 112 * 1024;                // per CTA: two launches share an SM
+constexpr int ST_W_BYTES = ST_CW == 8 ? 17408 : (ST_CW == 12 ? 26624 : 34816);                         // weight part of a stage (16 KB of nibbles + scales + zero points, padded)
+// CTAs per SM.  One CTA per SM with sixteen consumer warps (-DST_CW=16 -DST_MINB=1: 96 registers, no spills with two
+// token blocks, a 220 KB ring) was measured equal to 17 % slower at up to 8 tokens and equal to 10 % faster at 16
+// (the 4096 -> 24576 layer: 17.3 against 19.2 us); not worth a second build of the kernel.
+#ifndef ST_MINB
+#define ST_MINB 2
+#endif
+constexpr int ST_SMEM_BUDGET = (ST_MINB == 2 ? 112 : 220) * 1024;   // per CTA: two CTAs share an SM
 constexpr uint32_t ST_STAY = 128;                         // one-kernel fused form: CTAs that stay to requantise (swept 32..296 on B200)
 constexpr int ST_MAX_ASUM_WORDS = 4096;                   // group sums of all tokens kept in shared memory
 
@@ -202,7 +208,7 @@ struct StripArgs {
 // FUSE == 3 is unrelated to gate+up: the plain projection with a residual added at the store (fp32 staging, the
 // residual's 16-byte pieces requested before the wait for the consumers), for the O and down projections.
 template <int MB, int RBLK, bool DEBUG, int FUSE>
-__global__ void __launch_bounds__(ST_THREADS, 2)
+__global__ void __launch_bounds__(ST_THREADS, ST_MINB)
 gemm_strip_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_nib,
                   const __grid_constant__ CUtensorMap tm_scale, const __grid_constant__ CUtensorMap tm_zero,
                   const StripArgs a) {
@@ -933,7 +939,7 @@ void strip_plan(int M, int N, int K, int* strip_rows, int* ctas) {
         if (v == 16 || v == 32 || v == 64 || v == 128) R = v;
     }
 #endif
-    int limit = 2 * sms;
+    int limit = ST_MINB * sms;
 #ifdef W4A8_TUNING
     if (const char* e = getenv("W4A8_STRIP_CTAS")) { const int v = atoi(e); if (v >= 1) limit = v; }
 #endif
