@@ -121,9 +121,9 @@ w4a8_status w4a8_quantize_act(const void* x_bf16, int M, int K, int group,
  * between the cluster split-K kernel or the tcgen05 kernel, whichever a measured cost model predicts
  * faster for the shape (w4a8_plan tells which).
  * Results are run-to-run deterministic.
- * Programmatic dependent launch: w4a8_quantize_act and the weight-streaming kernels for up to 64
- * tokens are launched with programmatic stream serialisation (the tcgen05 kernel and the workspace
- * variant of the split-K kernel are launched plainly).  When consecutive library calls share a
+ * Programmatic dependent launch: w4a8_quantize_act, the weight-streaming kernels for up to 64
+ * tokens and the tensor-core kernel are launched with programmatic stream serialisation (only the
+ * workspace variant of the split-K kernel is launched plainly).  When consecutive library calls share a
  * stream, such a kernel may start, and prefetch packed weights, before its predecessor in the
  * stream has finished; it waits on the device before it reads any activation, token scale or group
  * sum, touches the workspace or writes any output.  packed_w is therefore the one argument that

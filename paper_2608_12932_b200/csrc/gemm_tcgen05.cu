@@ -133,6 +133,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                     int32_t* __restrict__ debug_partials, uint32_t* __restrict__ status,
                     int M, int N, int K, int m_tiles, int total_tiles, int S,
                     float* __restrict__ handover, uint32_t* __restrict__ handover_flags) {
+    // Programmatic dependent launch: the kernel after this one may start its prologue now; this one sets up tensor
+    // memory, barriers and its weight stream (weights never depend on the previous kernel) while its predecessor may
+    // still run, and the roles that touch activations, token scales, the workspace or the output wait below.
+    ptx::pdl_launch_dependents();
     using C = Cfg<TILE_M>;
     static_assert(!SPLIT || C::SB * C::B_BYTES >= TILE_M * TILE_N * 4 + 64, "the split-K exchange buffer lives in the activation ring");
     static_assert(!(SPLIT && PC), "the per-channel form is not split along K");
@@ -217,6 +221,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
         asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         if (warp == WARP_PRODUCER && lane == 0) {
             // ------------------------------------------------ producer: activation tiles ----
+            ptx::pdl_wait();                                    // the activations are the previous kernel's output
             uint32_t it = 0;
             bool ok = true;
             for (int si = 0; ok; ++si) {
@@ -385,6 +390,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
         else asm volatile("setmaxnreg.inc.sync.aligned.u32 160;");
         // --------------------------------------------------------------------- drain ----
         // Warp (q, h): TMEM lanes 32q..32q+31 (output channels), accumulator columns h*W.. (tokens).
+        ptx::pdl_wait();                                        // token scales, hand-over flags, residual and output
         const int q = warp & 3, h = (warp - WARP_DRAIN0) >> 2;
         const int n_local = q * 32 + lane;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + h * C::W;
@@ -658,6 +664,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
         __syncwarp();
     }
 
+    ptx::pdl_wait();                            // every thread, before the split-K tail's stores and the status word
     if (SPLIT) {
         // first barrier for every thread that has not passed it in the drain role, then the second one
         // (release after the pushes, acquire before the sums); this CTA then reduces its share of the tile
@@ -727,13 +734,15 @@ cudaError_t launch_tile(const int8_t* qa, const uint16_t* sa, const void* packed
     cfg.blockDim = dim3(TC_THREADS, 1, 1);
     cfg.dynamicSmemBytes = C::SMEM_ALLOC;
     cfg.stream = stream;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = SPLIT ? (unsigned)S : 1u;
-    attr.val.clusterDim.y = 1;
-    attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = SPLIT ? (unsigned)S : 1u;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<TILE_M, DEBUG, SPLIT, PC, BAL, RES>, tmap, tmap_y, static_cast<const uint8_t*>(packed), sa,
                               static_cast<__nv_bfloat16*>(y), static_cast<const __nv_bfloat16*>(residual), debug_partials,
                               reinterpret_cast<uint32_t*>(ws + WS_STATUS_OFF),
