@@ -89,13 +89,19 @@ struct Cfg {
     static constexpr int SB = TILE_M > 128 ? 5 : (TILE_M == 128 ? 6 : 8);     // activation stages
     static constexpr int SR = TILE_M > 128 ? 8 : (TILE_M == 128 ? 12 : 16);   // packed-blob stages: a short tile finishes a group
                                                                               // quickly, so more blobs must be in flight to cover HBM latency
-    static constexpr int SA_MAX = (TMEM_COLS - 2 * TILE_M) / A_COLS;
+// (four accumulator buffers at 64-row tiles, where tensor memory has the room, -DTC_NB64=4: same results, 0.5-2 % faster
+// - the MMA -> drain -> MMA round trip of a buffer is not what bounds the short-tile step)
+#ifndef TC_NB64
+#define TC_NB64 2
+#endif
+    static constexpr int NB = TILE_M == 64 ? TC_NB64 : 2;                      // accumulator buffers in flight
+    static constexpr int SA_MAX = (TMEM_COLS - NB * TILE_M) / A_COLS;
     static constexpr int SA = SA_MAX > 4 ? 4 : SA_MAX;                        // weight stages in TMEM
-    static constexpr int A_COL0 = 2 * TILE_M;                                 // first weight column (after two accumulators)
+    static constexpr int A_COL0 = NB * TILE_M;                                // first weight column (after the accumulators)
     static constexpr int B_OFF = 0;
     static constexpr int RAW_OFF = B_OFF + SB * B_BYTES;
     static constexpr int BAR_OFF = RAW_OFF + SR * RAW_STRIDE;
-    static constexpr int NUM_BARS = 2 * SR + SB + SA + 2 + DONE_RING + 2 + 2;
+    static constexpr int NUM_BARS = 2 * SR + SB + SA + 4 + DONE_RING + 2 + 2;
     static constexpr int MISC_OFF = (BAR_OFF + NUM_BARS * 8 + 15) & ~15;      // 16-byte aligned: staging is read with 16-byte loads
     static constexpr int W = TILE_M / 2;                                      // accumulator columns (tokens) per drain warp
     static constexpr int NCH = (W + 31) / 32;                                 // 32-column chunks per drain warp (the last may be 8 wide)
@@ -158,7 +164,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
     // one event frees the step's weight stage (unpack warps wait for step it - SA), its activation
     // stage (producer waits for step it - SB) and publishes its accumulator (drain warps wait for it).
     const int RAW_FULL = 0, RAW_EMPTY = C::SR, B_FULL = 2 * C::SR, A_FULL = B_FULL + C::SB, ACC_EMPTY = A_FULL + C::SA,
-              DONE = ACC_EMPTY + 2, FINAL = DONE + DONE_RING, TILE_DONE = FINAL + 2;
+              DONE = ACC_EMPTY + 4, FINAL = DONE + DONE_RING, TILE_DONE = FINAL + 2;
     auto done_bar = [&](uint32_t step) { return bar(DONE + (int)(step % DONE_RING)); };
     auto done_parity = [](uint32_t step) { return (step / DONE_RING) & 1u; };
     volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(smem + C::MISC_OFF);
@@ -173,7 +179,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
             }
             for (int i = 0; i < C::SB; ++i) ptx::mbar_init(bar(B_FULL + i), 1);
             for (int i = 0; i < C::SA; ++i) ptx::mbar_init(bar(A_FULL + i), NUM_UNPACK_WARPS);
-            for (int i = 0; i < 2; ++i) ptx::mbar_init(bar(ACC_EMPTY + i), NUM_DRAIN_WARPS);
+            for (int i = 0; i < 4; ++i) ptx::mbar_init(bar(ACC_EMPTY + i), NUM_DRAIN_WARPS);
             for (int i = 0; i < DONE_RING; ++i) ptx::mbar_init(bar(DONE + i), 1);
             for (int i = 0; i < 2; ++i) ptx::mbar_init(bar(FINAL + i), 1);
             for (int i = 0; i < 2; ++i) ptx::mbar_init(bar(TILE_DONE + i), 2);      // both MMA issuers
@@ -284,8 +290,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                 if (!segment(si, tile, gb, ge)) break;
                 // PC: both threads add into the buffer of the tile, which the drain warps left zeroed
                 // (integer sums commute, so the order of the two threads' MMAs does not matter)
-                const uint32_t buf = PC ? (tcount & 1u) : par;
-                const uint32_t d_tmem = tmem_u + buf * TILE_M;
+                uint32_t buf = PC ? (tcount & 1u) : par;
+                uint32_t d_tmem = tmem_u + buf * TILE_M;
                 bool mine = false;
                 for (int g = gb; g < ge; ++g, ++it) {
                     if ((it & 1u) != par) continue;
@@ -304,7 +310,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                         if (!(ok = ptx::mbar_wait(bar(B_FULL + sb), pb, abort_flag))) break;
                         if (!(ok = ptx::mbar_wait(bar(A_FULL + sa_), pas, abort_flag))) break;
                     }
-                    if (!(ok = ptx::mbar_wait(bar(ACC_EMPTY + buf), ((PC ? tcount : it) >> 1) & 1, abort_flag))) break;
+                    if (!PC && C::NB == 4) { buf = it & 3u; d_tmem = tmem_u + buf * TILE_M; }      // this issuer's two buffers in turn
+                    if (!(ok = ptx::mbar_wait(bar(ACC_EMPTY + buf), (PC ? (tcount >> 1) : (it / C::NB)) & 1, abort_flag))) break;
                     ptx::tc_fence_after_sync();
                     const uint64_t bd = b_desc0 + (uint64_t)(sb * (C::B_BYTES / 16));
                     const uint32_t a_tmem = tmem_u + C::A_COL0 + sa_ * A_COLS;
@@ -406,9 +413,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
             ptx::tc_fence_before_sync();
             __syncwarp();
         }
-        if (lane == 0) {                                          // both accumulator buffers start out free
-            ptx::mbar_arrive(bar(ACC_EMPTY + 0));
-            ptx::mbar_arrive(bar(ACC_EMPTY + 1));
+        if (lane == 0) {                                          // the accumulator buffers start out free
+            for (int i = 0; i < 4; ++i) ptx::mbar_arrive(bar(ACC_EMPTY + i));
         }
         uint32_t it = 0, tcount = 0;
         bool ok = true;
@@ -494,7 +500,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_qa, const __grid_co
                 }
             }
             for (int g = gb; g < (PC ? gb : ge); ++g, ++it) {
-                const uint32_t buf = it & 1;
+                const uint32_t buf = it & (C::NB - 1);
                 const float sw = __half2float(__ushort_as_half(sw_bits));
                 if (g + 1 < ge) sw_bits = __ldg(reinterpret_cast<const uint16_t*>(sw_ptr + (size_t)(g + 1) * BLOB_BYTES));
                 // (short tiles: this warp mostly waits, and a polling loop's probes queue up in front of the unpack
